@@ -1,0 +1,623 @@
+/*
+ * BalanceRoute reference checker -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, single-threaded restatement of the routing step as the paper
+ * defines it, used only to check the CUDA library and to be timed as a CPU
+ * baseline.  It shares no code with the CUDA path.  Integer quantities are
+ * int64; horizon scores are fp64 evaluated term by term in the order the
+ * formulas are written (compile with -ffp-contract=off).
+ *
+ * Passages followed:
+ *   workload model (loads s_i + j - 1, active sets, capacity B) ... Section 2.2
+ *   imbalance I(k) = G M(k) - sum_g L_g(k), safe margin m_g ...... Section 3.1
+ *   F-score of BR-0 ............................................... Eq. 1
+ *   two-stage BR-0 (greedy fill, refined allocation, guard) ....... Section 3.2, Algorithm 1
+ *   horizon F-score of BR-H ....................................... Eq. 2
+ *   two-stage BR-H ................................................ Section 4.2, Algorithm 2
+ *   c_hat from classifier output, composite and clip .............. Eqs. 3-5
+ *   horizon projection, envelope, margin vectors .................. Eq. 6 and the paragraph after it
+ *   refresh period, confidence gate, floor ........................ Appendix "Refresh logic"
+ *   exhaustive subset enumeration over the R_max window ........... Appendix "Bit-set subset selection"
+ *   round-robin and least-loaded comparison routers ............... Section 5.1 "Baselines"
+ *
+ * Readings taken where the paper is silent or ambiguous are marked READING
+ * below.  Functions whose tie-break choices have no counterpart in the paper
+ * are "parity unpinned" against the paper in that respect only: orc_step's
+ * tie-breaks (worker ties, request ties, subset ties) and slot placement.
+ * Everything else is pinned by the tests under tests/ (closed forms of Eq. 1,
+ * the identity F = -Delta I, the H = 0 reduction, Eq. 4, brute force).
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+#define ORC_EMPTY INT32_MIN
+
+typedef struct {
+    int32_t G, H, B, W, R_max, S_greedy;
+    double  alpha, beta, gamma;
+    int32_t delta_T;
+    float   gate, c_floor;
+    int32_t score_mode;          /* 0: Eq. 1 in integers; 1: Eq. 2 in fp64          */
+    int32_t term_mode;           /* 0 none; 1 constant hazard; 2 Bernoulli(probs[.][0]) */
+    uint32_t hazard_thr;
+    const uint32_t *arr_cdf;     /* [arr_period][arr_len] rows for this instance    */
+    int32_t arr_len, arr_period;
+    const int32_t *len_tab;
+    int32_t len_tab_log2;
+    int32_t burst_every, burst_size;
+    int32_t router;              /* 0 BalanceRoute; 1 round-robin; 2 least-loaded   */
+} orc_params;
+
+typedef struct {
+    orc_params p;
+    uint64_t seed;
+    int32_t  k;
+    uint32_t next_id;
+    int32_t  rr_ptr;
+    /* one entry per slot (g * B + b) */
+    uint8_t  *occ;
+    uint32_t *sid;
+    int64_t  *cur;
+    float    *chat;
+    int32_t  *tau;
+    /* waiting requests in arrival order */
+    int32_t  *qs;
+    uint32_t *qid;
+    uint8_t  *qgone;
+    int32_t  qn;
+    /* round state */
+    int64_t *Lh, *Mh, *m;        /* [G][H+1], [H+1], [G][H+1] */
+    int32_t *cap;
+    double  *d;
+    double   D;
+    /* counters since creation */
+    int64_t dropped, admitted, s1_iters, s2_pops, guard_hits;
+} orc_inst;
+
+/* ------------------------------------------------------------------ */
+/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): ten rounds of   */
+/* two 32x32->64 multiplies with a Weyl key schedule.                  */
+/* ------------------------------------------------------------------ */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2 };
+
+static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
+{
+    /* counter = (step, entity / 4, stream, 0); word entity % 4 of the block */
+    uint32_t ctr[4] = { (uint32_t)s->k, entity >> 2, stream, 0u };
+    uint32_t key[2] = { (uint32_t)s->seed, (uint32_t)(s->seed >> 32) };
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return out[entity & 3u];
+}
+
+/* ------------------------------------------------------------------ */
+/* scores                                                              */
+/* ------------------------------------------------------------------ */
+
+/* Eq. 1: F_g(Q) = Delta - G (Delta - m_g)_+ */
+int64_t orc_f_br0(int32_t G, int64_t delta, int64_t m)
+{
+    int64_t over = delta - m;
+    if (over < 0) over = 0;
+    return delta - (int64_t)G * over;
+}
+
+/* d = (1, gamma, ..., gamma^H) by repeated multiplication; returns 1^T d */
+double orc_discount(int32_t H, double gamma, double *d)
+{
+    double D = 0.0;
+    for (int h = 0; h <= H; ++h) {
+        d[h] = (h == 0) ? 1.0 : d[h - 1] * gamma;
+        D = D + d[h];
+    }
+    return D;
+}
+
+/* Eq. 2: F_g(Q) = alpha (1^T d) Delta - beta (Delta 1 - m_g)_+^T d */
+double orc_f_brh(int32_t H, double alpha, double beta, const double *d, double D,
+                 int64_t delta, const int64_t *m)
+{
+    double pen = 0.0;
+    for (int h = 0; h <= H; ++h) {
+        int64_t over = delta - m[h];
+        if (over < 0) over = 0;
+        pen = pen + d[h] * (double)over;
+    }
+    return (alpha * D) * (double)delta - beta * pen;
+}
+
+/* total imbalance I = G max L - sum L (Section 3.1) */
+int64_t orc_imbalance(int32_t G, const int64_t *L)
+{
+    int64_t M = L[0], S = 0;
+    for (int g = 0; g < G; ++g) { if (L[g] > M) M = L[g]; S += L[g]; }
+    return (int64_t)G * M - S;
+}
+
+/*
+ * Eqs. 3-5 from per-horizon-step hazards q_1..q_H (READING: q_h is the
+ * probability of finishing at in-window step h given alive entering it):
+ *   P(r = h) = q_h prod_{j<h} (1 - q_j),  p_fin = 1 - prod_{h<=H} (1 - q_h),
+ *   E[min(r, H)] = sum_{h=1..H} prod_{j<h} (1 - q_j)      (tail-sum form),
+ * which equals (1 - p_fin) H + p_fin mu_rem of Eq. 4.  Not clipped here.
+ */
+double orc_chat_star(int32_t H, const float *q, double *p_fin)
+{
+    double surv = 1.0, c = 0.0;
+    for (int h = 0; h < H; ++h) {
+        c = c + surv;
+        surv = surv * (1.0 - (double)q[h]);
+    }
+    if (p_fin) *p_fin = 1.0 - surv;
+    return c;
+}
+
+/* the same expectation written as Eq. 4 / Eq. 5: (1 - p) H + p mu_rem */
+double orc_chat_two_stage(int32_t H, const float *q, double *p_fin, double *mu_rem)
+{
+    double surv = 1.0, p = 0.0, num = 0.0;
+    for (int h = 1; h <= H; ++h) {
+        double ph = surv * (double)q[h - 1];      /* P(r = h) */
+        p += ph;
+        num += ph * (double)h;
+        surv *= 1.0 - (double)q[h - 1];
+    }
+    double mu = (p > 0.0) ? num / p : (double)H;
+    if (p_fin) *p_fin = p;
+    if (mu_rem) *mu_rem = mu;
+    return (1.0 - p) * (double)H + p * mu;
+}
+
+/* ------------------------------------------------------------------ */
+/* instance life cycle                                                 */
+/* ------------------------------------------------------------------ */
+orc_inst *orc_create(const orc_params *p, uint64_t seed)
+{
+    orc_inst *s = (orc_inst *)calloc(1, sizeof(orc_inst));
+    s->p = *p;
+    s->seed = seed;
+    int A = p->G * p->B, H1 = p->H + 1;
+    s->occ = (uint8_t *)calloc(A, 1);
+    s->sid = (uint32_t *)calloc(A, sizeof(uint32_t));
+    s->cur = (int64_t *)calloc(A, sizeof(int64_t));
+    s->chat = (float *)calloc(A, sizeof(float));
+    s->tau = (int32_t *)calloc(A, sizeof(int32_t));
+    s->qs = (int32_t *)calloc(p->W, sizeof(int32_t));
+    s->qid = (uint32_t *)calloc(p->W, sizeof(uint32_t));
+    s->qgone = (uint8_t *)calloc(p->W, 1);
+    s->Lh = (int64_t *)calloc((size_t)p->G * H1, sizeof(int64_t));
+    s->Mh = (int64_t *)calloc(H1, sizeof(int64_t));
+    s->m = (int64_t *)calloc((size_t)p->G * H1, sizeof(int64_t));
+    s->cap = (int32_t *)calloc(p->G, sizeof(int32_t));
+    s->d = (double *)calloc(H1, sizeof(double));
+    s->D = orc_discount(p->H, p->gamma, s->d);
+    return s;
+}
+
+void orc_destroy(orc_inst *s)
+{
+    if (!s) return;
+    free(s->occ); free(s->sid); free(s->cur); free(s->chat); free(s->tau);
+    free(s->qs); free(s->qid); free(s->qgone);
+    free(s->Lh); free(s->Mh); free(s->m); free(s->cap); free(s->d);
+    free(s);
+}
+
+/* act_base[slot] = cur - k for an occupied slot, ORC_EMPTY otherwise */
+void orc_set_state(orc_inst *s, int32_t k, uint32_t next_id,
+                   const int32_t *act_base, const uint32_t *act_id,
+                   const float *chat, const int32_t *tau,
+                   const int32_t *qs, const uint32_t *qid, int32_t qn)
+{
+    int A = s->p.G * s->p.B;
+    s->k = k; s->next_id = next_id;
+    for (int a = 0; a < A; ++a) {
+        s->occ[a] = act_base[a] != ORC_EMPTY;
+        s->cur[a] = s->occ[a] ? (int64_t)act_base[a] + k : 0;
+        s->sid[a] = act_id ? act_id[a] : 0u;
+        s->chat[a] = chat ? chat[a] : (float)s->p.H;
+        s->tau[a] = tau ? tau[a] : 0;
+    }
+    s->qn = qn;
+    for (int i = 0; i < qn; ++i) { s->qs[i] = qs[i]; s->qid[i] = qid ? qid[i] : 0u; }
+}
+
+void orc_get_state(const orc_inst *s, int32_t *k, uint32_t *next_id,
+                   int32_t *act_base, uint32_t *act_id, float *chat, int32_t *tau,
+                   int32_t *qs, uint32_t *qid, int32_t *qn, int64_t *counters)
+{
+    int A = s->p.G * s->p.B;
+    *k = s->k; *next_id = s->next_id;
+    for (int a = 0; a < A; ++a) {
+        act_base[a] = s->occ[a] ? (int32_t)(s->cur[a] - s->k) : ORC_EMPTY;
+        if (act_id) act_id[a] = s->sid[a];
+        if (chat) chat[a] = s->chat[a];
+        if (tau) tau[a] = s->tau[a];
+    }
+    *qn = s->qn;
+    for (int i = 0; i < s->qn; ++i) { qs[i] = s->qs[i]; if (qid) qid[i] = s->qid[i]; }
+    if (counters) {
+        counters[0] = s->dropped; counters[1] = s->admitted; counters[2] = s->s1_iters;
+        counters[3] = s->s2_pops; counters[4] = s->guard_hits;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* one decode step                                                     */
+/* ------------------------------------------------------------------ */
+
+/* a0: prefill-completed requests join R_wait in arrival order */
+static void arrive(orc_inst *s)
+{
+    const orc_params *p = &s->p;
+    uint32_t u = draw(s, 0u, STREAM_ARR_COUNT);
+    const uint32_t *row = p->arr_cdf + (size_t)(s->k % p->arr_period) * p->arr_len;
+    int32_t n = 0;
+    for (int j = 0; j < p->arr_len; ++j) if (u >= row[j]) ++n;
+    if (p->burst_every > 0 && s->k > 0 && s->k % p->burst_every == 0) n += p->burst_size;
+    for (int32_t j = 0; j < n; ++j) {
+        uint32_t r = draw(s, (uint32_t)j, STREAM_ARR_LEN);
+        int32_t len = p->len_tab[r >> (32 - p->len_tab_log2)];
+        if (s->qn < p->W) {
+            s->qs[s->qn] = len;
+            s->qid[s->qn] = s->next_id + (uint32_t)j;
+            s->qn++;
+        } else {
+            s->dropped++;
+        }
+    }
+    s->next_id += (uint32_t)n;     /* READING: ids are consumed by dropped arrivals too */
+}
+
+/* a1: c_hat maintenance (refresh period, gate, floor) */
+static void predict(orc_inst *s, const float *probs)
+{
+    const orc_params *p = &s->p;
+    int A = p->G * p->B;
+    if (p->H == 0) return;
+    for (int a = 0; a < A; ++a) {
+        if (!s->occ[a]) continue;
+        int32_t t = s->tau[a] + 1;
+        float c = s->chat[a] - 1.0f;               /* one step less of in-window work */
+        if (t >= p->delta_T || c < p->c_floor) {   /* periodic, or floor crossed      */
+            double p_fin;
+            double cs = orc_chat_star(p->H, probs + (size_t)a * p->H, &p_fin);
+            double v;
+            if (p_fin >= (double)p->gate) {
+                v = cs;
+                if (v < (double)p->c_floor) v = (double)p->c_floor;
+                if (v > (double)p->H) v = (double)p->H;
+            } else {
+                v = (double)p->H;                  /* gate closed: conservative anchor */
+            }
+            s->chat[a] = (float)v;
+            s->tau[a] = 0;
+        } else {
+            s->chat[a] = c;
+            s->tau[a] = t;
+        }
+    }
+}
+
+/* Eq. 6 and the margin-vector paragraph: L_g(k+h), envelope M_h, margins.
+ * READING: offsets h = 0..H; a running request contributes cur + h at offset h
+ * iff h = 0 or h <= c_hat, so offset 0 is L_g(k). */
+static void margins(orc_inst *s)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    for (int h = 0; h < H1; ++h) {
+        int64_t M = s->Lh[h];
+        for (int g = 1; g < p->G; ++g) if (s->Lh[g * H1 + h] > M) M = s->Lh[g * H1 + h];
+        s->Mh[h] = M;
+        for (int g = 0; g < p->G; ++g) {
+            int64_t v = M - s->Lh[g * H1 + h];
+            s->m[g * H1 + h] = v > 0 ? v : 0;
+        }
+    }
+}
+
+static void project(orc_inst *s)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    for (int g = 0; g < p->G; ++g) {
+        int n = 0;
+        for (int h = 0; h < H1; ++h) s->Lh[g * H1 + h] = 0;
+        for (int b = 0; b < p->B; ++b) {
+            int a = g * p->B + b;
+            if (!s->occ[a]) continue;
+            ++n;
+            for (int h = 0; h < H1; ++h)
+                if (h == 0 || (float)h <= s->chat[a]) s->Lh[g * H1 + h] += s->cur[a] + h;
+        }
+        s->cap[g] = p->B - n;
+    }
+    margins(s);
+}
+
+static double score(const orc_inst *s, int g, int64_t delta)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    if (p->score_mode == 0)
+        return (double)orc_f_br0(p->G, delta, s->m[g * H1]);   /* exact: |F| < 2^53 */
+    return orc_f_brh(p->H, p->alpha, p->beta, s->d, s->D, delta, s->m + g * H1);
+}
+
+/* argmax_i F_g({i}) over all of R_wait; ties -> earliest arrival */
+static int best_single(const orc_inst *s, int g)
+{
+    int best = -1; double fb = 0.0;
+    for (int i = 0; i < s->qn; ++i) {
+        if (s->qgone[i]) continue;
+        double f = score(s, g, s->qs[i]);
+        if (best < 0 || f > fb) { best = i; fb = f; }
+    }
+    return best;
+}
+
+/* sticky admission of queue entry i to worker g (lowest free slot) */
+static void commit(orc_inst *s, int i, int g, int32_t *assign)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1, b = 0;
+    while (s->occ[g * p->B + b]) ++b;
+    int a = g * p->B + b;
+    s->occ[a] = 1; s->sid[a] = s->qid[i]; s->cur[a] = s->qs[i];     /* w^(1) = s_i */
+    s->chat[a] = (float)p->H;
+    s->tau[a] = p->delta_T - 1;           /* READING: first prediction at the next step */
+    s->qgone[i] = 1;
+    s->cap[g]--;
+    /* READING: the admitted request adds a constant s_i at every offset */
+    for (int h = 0; h < H1; ++h) s->Lh[g * H1 + h] += s->qs[i];
+    margins(s);
+    if (assign) assign[i] = a;
+    s->admitted++;
+}
+
+static int64_t waiting(const orc_inst *s)
+{
+    int64_t n = 0;
+    for (int i = 0; i < s->qn; ++i) n += !s->qgone[i];
+    return n;
+}
+
+static void route_balance(orc_inst *s, int32_t *assign)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    int64_t S_tot = 0;
+    for (int g = 0; g < p->G; ++g) S_tot += s->cap[g];
+    if (S_tot == 0 || s->qn == 0) return;
+
+    /* Stage 1: greedy fill */
+    while (S_tot > p->S_greedy && waiting(s) > 0) {
+        int g = 0;     /* most free slots; ties -> smallest L_g(k); then lowest g */
+        for (int x = 1; x < p->G; ++x)
+            if (s->cap[x] > s->cap[g] ||
+                (s->cap[x] == s->cap[g] && s->Lh[x * H1] < s->Lh[g * H1])) g = x;
+        int i = best_single(s, g);
+        commit(s, i, g, assign);
+        S_tot--;
+        s->s1_iters++;
+    }
+
+    /* Stage 2: refined allocation.  READING: the priority queue is read with
+     * current keys at every pop (largest cap, then largest margin / horizon-min
+     * margin, then lowest g), which is what "reinsert" with updated margins gives. */
+    for (;;) {
+        if (waiting(s) == 0) break;
+        int g = -1; int64_t keyg = 0;
+        for (int x = 0; x < p->G; ++x) {
+            if (s->cap[x] <= 0) continue;
+            int64_t key = s->m[x * H1];
+            for (int h = 1; h < H1; ++h) if (s->m[x * H1 + h] < key) key = s->m[x * H1 + h];
+            if (g < 0 || s->cap[x] > s->cap[g] || (s->cap[x] == s->cap[g] && key > keyg)) {
+                g = x; keyg = key;
+            }
+        }
+        if (g < 0) break;
+        s->s2_pops++;
+
+        /* window: the R_max largest waiting requests (READING: sorted by s_i
+         * descending, ties by arrival order) */
+        int win[32], nw = 0;
+        for (int r = 0; r < p->R_max; ++r) {
+            int best = -1;
+            for (int i = 0; i < s->qn; ++i) {
+                if (s->qgone[i]) continue;
+                int taken = 0;
+                for (int j = 0; j < nw; ++j) taken |= (win[j] == i);
+                if (taken) continue;
+                if (best < 0 || s->qs[i] > s->qs[best]) best = i;
+            }
+            if (best < 0) break;
+            win[nw++] = best;
+        }
+        int lim = s->cap[g] < p->R_max ? s->cap[g] : p->R_max;
+        uint32_t best_mask = 0; double fb = 0.0;
+        for (uint32_t mask = 1; mask < (1u << nw); ++mask) {
+            if (__builtin_popcount(mask) > lim) continue;
+            int64_t delta = 0;
+            for (int j = 0; j < nw; ++j) if (mask >> j & 1u) delta += s->qs[win[j]];
+            double f = score(s, g, delta);
+            if (best_mask == 0 || f > fb) { best_mask = mask; fb = f; }
+        }
+        if (fb <= 0.0) {
+            /* starvation guard.  READING: least-bad single request of all of R_wait */
+            s->guard_hits++;
+            commit(s, best_single(s, g), g, assign);
+        } else {
+            for (int j = 0; j < nw; ++j)
+                if (best_mask >> j & 1u) commit(s, win[j], g, assign);
+        }
+    }
+}
+
+/* comparison routers over the same arrivals and terminations */
+static void route_round_robin(orc_inst *s, int32_t *assign)
+{
+    const orc_params *p = &s->p;
+    for (int i = 0; i < s->qn; ++i) {
+        int g = -1;
+        for (int t = 0; t < p->G; ++t) {
+            int x = (s->rr_ptr + t) % p->G;
+            if (s->cap[x] > 0) { g = x; break; }
+        }
+        if (g < 0) break;
+        commit(s, i, g, assign);
+        s->rr_ptr = (g + 1) % p->G;
+    }
+}
+
+static void route_least_loaded(orc_inst *s, int32_t *assign)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    for (int i = 0; i < s->qn; ++i) {
+        int g = -1;
+        for (int x = 0; x < p->G; ++x)
+            if (s->cap[x] > 0 && (g < 0 || s->Lh[x * H1] < s->Lh[g * H1])) g = x;
+        if (g < 0) break;
+        commit(s, i, g, assign);
+    }
+}
+
+/*
+ * One decode step k:  ARRIVE -> PREDICT -> ROUTE -> RECORD -> ADVANCE.
+ *   probs   [G*B][H] classifier output for this step (NULL if unused)
+ *   assign  [W]  slot index g*B+b per queue position as of after ARRIVE, -1 if kept waiting
+ *   load    [G]  L_g(k) after admissions
+ *   trace   [3]  (max_g L_g, min_g L_g, sum_g L_g)
+ *   fscore  [W][G] optional: F_g({i}) before the first admission
+ */
+void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
+              int64_t *trace, double *fscore)
+{
+    const orc_params *p = &s->p;
+    int A = p->G * p->B;
+
+    arrive(s);
+    predict(s, probs);
+    project(s);
+
+    for (int i = 0; i < p->W; ++i) { assign[i] = -1; s->qgone[i] = 0; }
+    if (fscore) {
+        for (int i = 0; i < p->W; ++i)
+            for (int g = 0; g < p->G; ++g)
+                fscore[(size_t)i * p->G + g] = (i < s->qn) ? score(s, g, s->qs[i]) : 0.0;
+    }
+
+    if (p->router == 0) route_balance(s, assign);
+    else if (p->router == 1) route_round_robin(s, assign);
+    else route_least_loaded(s, assign);
+
+    /* stable removal of admitted requests */
+    int w = 0;
+    for (int i = 0; i < s->qn; ++i)
+        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; ++w; }
+    s->qn = w;
+
+    /* RECORD: loads from scratch */
+    int64_t mx = 0, mn = 0, sum = 0;
+    for (int g = 0; g < p->G; ++g) {
+        int64_t L = 0;
+        for (int b = 0; b < p->B; ++b) if (s->occ[g * p->B + b]) L += s->cur[g * p->B + b];
+        load[g] = L;
+        if (g == 0 || L > mx) mx = L;
+        if (g == 0 || L < mn) mn = L;
+        sum += L;
+    }
+    trace[0] = mx; trace[1] = mn; trace[2] = sum;
+
+    /* ADVANCE: every running request, the just-admitted ones included, either
+     * finishes at the end of this step or grows by one token */
+    for (int a = 0; a < A; ++a) {
+        if (!s->occ[a]) continue;
+        int fin = 0;
+        if (p->term_mode == 1) {
+            fin = draw(s, (uint32_t)a, STREAM_TERM) < p->hazard_thr;
+        } else if (p->term_mode == 2) {
+            uint32_t u = draw(s, (uint32_t)a, STREAM_TERM) >> 8;       /* 24 bits */
+            fin = ((float)u * 5.9604644775390625e-8f) < probs[(size_t)a * p->H];
+        }
+        if (fin) { s->occ[a] = 0; s->cur[a] = 0; }
+        else s->cur[a] += 1;
+    }
+    s->k += 1;
+}
+
+/* ------------------------------------------------------------------ */
+/* helpers exposed for the tests                                       */
+/* ------------------------------------------------------------------ */
+
+/* best subset of a window by exhaustive enumeration; returns its mask */
+uint32_t orc_best_subset(int32_t score_mode, int32_t G, int32_t H, double alpha, double beta,
+                         double gamma, const int64_t *m, const int32_t *win, int32_t nw,
+                         int32_t lim, double *f_out)
+{
+    double d[65]; double D = orc_discount(H, gamma, d);
+    uint32_t best_mask = 0; double fb = 0.0;
+    for (uint32_t mask = 1; mask < (1u << nw); ++mask) {
+        if (__builtin_popcount(mask) > lim) continue;
+        int64_t delta = 0;
+        for (int j = 0; j < nw; ++j) if (mask >> j & 1u) delta += win[j];
+        double f = score_mode == 0 ? (double)orc_f_br0(G, delta, m[0])
+                                   : orc_f_brh(H, alpha, beta, d, D, delta, m);
+        if (best_mask == 0 || f > fb) { best_mask = mask; fb = f; }
+    }
+    if (f_out) *f_out = fb;
+    return best_mask;
+}
+
+/* ROUTE phase alone on a given snapshot (no arrivals, no advance): used by the
+ * brute-force and invariant tests.  loads_out gets L_g after admissions. */
+void orc_route_only(orc_inst *s, int32_t *assign, int64_t *loads_out)
+{
+    const orc_params *p = &s->p;
+    int H1 = p->H + 1;
+    project(s);
+    for (int i = 0; i < p->W; ++i) { assign[i] = -1; s->qgone[i] = 0; }
+    if (p->router == 0) route_balance(s, assign);
+    else if (p->router == 1) route_round_robin(s, assign);
+    else route_least_loaded(s, assign);
+    for (int g = 0; g < p->G; ++g) loads_out[g] = s->Lh[g * H1];
+    int w = 0;
+    for (int i = 0; i < s->qn; ++i)
+        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; ++w; }
+    s->qn = w;
+}
+
+/* projected loads of the current snapshot: Lh [G][H+1], Mh [H+1], m [G][H+1] */
+void orc_projection(orc_inst *s, int64_t *Lh, int64_t *Mh, int64_t *m)
+{
+    int n = s->p.G * (s->p.H + 1);
+    project(s);
+    memcpy(Lh, s->Lh, n * sizeof(int64_t));
+    memcpy(Mh, s->Mh, (s->p.H + 1) * sizeof(int64_t));
+    memcpy(m, s->m, n * sizeof(int64_t));
+}
+
+/* PREDICT alone (for the refresh-rule tests) */
+void orc_predict_only(orc_inst *s, const float *probs) { predict(s, probs); }
