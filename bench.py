@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the BalanceRoute routing step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A "step" is one launch of the whole routing path (ARRIVE, PREDICT, ROUTE, RECORD, ADVANCE)
+over one batch of 4,096 independent BR-0 instances (G = 32, 256 waiting each: the batched
+HBM-throughput configuration).  Several instance sets are stepped in rotation so that the
+data touched between two visits of the same set exceeds the L2 cache.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_06113_b200 import workload as wlm  # noqa: E402
+
+METRIC = "routing instance-steps/sec (batched BR-0, 4096 instances, G=32, W=256)"
+UNIT = "instance-steps/s"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
+    """Bytes one instance-step has to move once: running-request state in, queue in,
+    assignments out, per-worker state in and out, slot edits."""
+    A, G, W, H = cfg.G * cfg.B, cfg.G, cfg.W, cfg.H
+    b = 4.0 * A + 8.0 * W + 4.0 * W + 20.0 * G + 28.0 * G + 24.0 + 8.0 * edits_per_step
+    if H > 0:
+        b += 5.0 * A + 4.0 * H * A * rho + 5.0 * A / cfg.delta_T
+    return b
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except Exception:
+                self.p.kill()
+        try:
+            self.f.flush()
+            rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+            sm = [float(r[1]) for r in rows if len(r) >= 9]
+            if sm:
+                out["sm_mhz"] = float(np.median(sm))
+                out["sm_max_mhz"] = float(rows[0][2])
+                out["samples"] = len(sm)
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                for j, n in enumerate(names):
+                    if any(r[5 + j].strip().lower() == "active" for r in rows if len(r) >= 9):
+                        out["reasons"].append(n)
+            os.unlink(self.f.name)
+        except Exception:
+            pass
+        return out
+
+
+def dist_setup(args):
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        if args.impl == "reference":
+            return world, rank, local, None
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        return world, rank, local, dist
+    return world, rank, local, None
+
+
+# ----------------------------------------------------------------------------- CPU arm
+def oracle_rate(cfg_name: str, budget_s: float, n_inst: int, max_steps: int):
+    """Instance-steps/s of the CPU checker, single thread, on the first n_inst instances."""
+    import oracle
+    cfg = wlm.get_config(cfg_name)
+    wl = wlm.make_workload(cfg, n_instances=n_inst)
+    orcs = [oracle.instance_from_workload(wl, i) for i in range(n_inst)]
+    probs = [wlm.term_probs_np(wl, k) for k in range(min(max_steps, 8))] if cfg.H > 0 else None
+    done = 0
+    t0 = time.perf_counter()
+    for k in range(max_steps):
+        for i, o in enumerate(orcs):
+            o.step(None if probs is None else probs[k % len(probs)][i])
+        done += n_inst
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return done / dt, done, dt
+
+
+def run_reference(args):
+    """The CPU checker as it stands, timed on host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfg = wlm.get_config("c3")
+    n_inst = 32
+    wl = wlm.make_workload(cfg, n_instances=n_inst)
+    orcs = [oracle.instance_from_workload(wl, i) for i in range(n_inst)]
+    for _ in range(args.warmup):
+        for o in orcs:
+            o.step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for o in orcs:
+            o.step()
+    dt = time.perf_counter() - t0
+    val = n_inst * args.steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+        "data": "synthetic",
+        "config": {"workload": "c3 (BR-0 batched, G=32, B=64, W=256), 32-instance sample per step"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{n_inst} instances x {args.steps} steps of c3, single thread"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+class RotatingSets:
+    """R independent instance sets of one configuration, stepped in rotation."""
+
+    def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=0):
+        import torch
+        from paper_2605_06113_b200.binding import Router
+        self.torch = torch
+        self.cfg = wlm.get_config(cfg_name)
+        self.N = n_inst
+        self.sets = []
+        self.router = None
+        for r in range(n_sets):
+            wl = wlm.make_workload(self.cfg, n_instances=n_inst, first_instance=seed_offset + r * n_inst)
+            if self.router is None:
+                self.wl0 = wl
+                self.router = Router(wl, device=device, threads=threads)
+                arr_rows = [wl.arr_cdf]
+            elif wl.arr_inst_stride:
+                arr_rows.append(wl.arr_cdf)
+            self.sets.append(dict(wl=wl, st=None))
+        # per-instance arrival rows of all sets live in one table; set r starts at row r * N
+        if self.wl0.arr_inst_stride:
+            from paper_2605_06113_b200 import binding
+            import ctypes as C
+            table = np.concatenate(arr_rows, axis=0)
+            self.router.close()
+            big = self.sets[0]["wl"]
+            big_tab = wlm.Workload(cfg=big.cfg, seeds=big.seeds, len_tab=big.len_tab, beta_tab=big.beta_tab,
+                                   arr_cdf=table, arr_period=big.arr_period,
+                                   arr_inst_stride=big.arr_inst_stride, hazard_thr=big.hazard_thr,
+                                   state=big.state)
+            self.router = Router(big_tab, device=device, threads=threads)
+        # all sets share one allocation per array so that `first_instance` selects the set
+        keys = list(self.sets[0]["wl"].state.keys())
+        cat = {k: np.concatenate([s["wl"].state[k] for s in self.sets], axis=0) for k in keys}
+        self.st = self.router.device_state(cat)
+        self.out = self.router.outputs(n_inst * n_sets)
+        self.out = {k: v[0] for k, v in self.out.items()}      # [R*N, ...]
+        self.out_view = {k: v.unsqueeze(0) for k, v in self.out.items()}
+        self.probs = None
+        if self.cfg.H > 0:
+            ring = max(1, probs_ring)
+            seeds_t = torch.from_numpy(np.concatenate([s["wl"].seeds for s in self.sets]).astype(np.int64)).to(device)
+            tab_t = torch.from_numpy(self.wl0.beta_tab).to(device)
+            self.probs = []
+            for j in range(ring):
+                self.probs.append(wlm.term_probs_torch(self.wl0, j, device, seeds_t=seeds_t, tab_t=tab_t).contiguous())
+        self.n_sets = n_sets
+        self.launch = 0
+
+    def step(self):
+        r = self.launch % self.n_sets
+        probs = None
+        if self.probs is not None:
+            probs = self.probs[(self.launch // self.n_sets) % len(self.probs)]
+        self.router.step(self.st, self.out_view, probs, N=self.N, first=r * self.N)
+        self.launch += 1
+
+
+def time_launches(torch, fn, warmup, steps, dist=None):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        torch.cuda.synchronize()
+        ms = float(t.item())
+    return ms
+
+
+def latency_path(torch, cfg_name, device, steps, overrides=None):
+    """Single instance, graph-replayed step: host-observed and device latency per step."""
+    from paper_2605_06113_b200.binding import Router
+    cfg = wlm.get_config(cfg_name, **(overrides or {}))
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device=device)
+    st = r.device_state()
+    out = r.outputs(1)
+    probs = None
+    seeds_t = tab_t = None
+    if cfg.H > 0:
+        seeds_t = torch.from_numpy(wl.seeds.astype(np.int64)).to(device)
+        tab_t = torch.from_numpy(wl.beta_tab).to(device)
+        probs = wlm.term_probs_torch(wl, 0, device, seeds_t=seeds_t, tab_t=tab_t).contiguous()
+    r.graph_capture(st, out, probs)
+    host_us, dev_us = [], []
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    for k in range(steps):
+        if cfg.H > 0:
+            wlm.term_probs_torch(wl, k, device, seeds_t=seeds_t, tab_t=tab_t, out=probs)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record()
+        r.graph_step()
+        e1.record()
+        torch.cuda.synchronize()
+        host_us.append(1e6 * (time.perf_counter() - t0))
+        dev_us.append(1e3 * e0.elapsed_time(e1))
+    r.close()
+    h = np.array(host_us[20:]); d = np.array(dev_us[20:])
+    return {"workload": cfg_name, "G": cfg.G, "W": cfg.W, "H": cfg.H, "steps": steps,
+            "host_p50_us": float(np.percentile(h, 50)), "host_p95_us": float(np.percentile(h, 95)),
+            "host_p99_us": float(np.percentile(h, 99)), "device_p50_us": float(np.percentile(d, 50)),
+            "device_p99_us": float(np.percentile(d, 99))}
+
+
+def run_ours(args):
+    import torch
+    world, rank, local, dist = dist_setup(args)
+    device = f"cuda:{local}"
+    torch.cuda.set_device(local)
+    peak, peak_kind = measured_peaks()
+
+    # ---------------- headline: c3 batched ----------------
+    cfg = wlm.get_config("c3")
+    N = cfg.N
+    per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
+    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
+    sets = RotatingSets("c3", N, n_sets, device, seed_offset=rank * n_sets * N, threads=args.threads)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms = time_launches(torch, sets.step, args.warmup, args.steps, dist)
+    clocks = sampler.stop()
+    cnt = sets.out["counters"].to(torch.float64).view(n_sets, N, 4).mean(dim=(0, 1)).cpu().numpy()
+    bad = int((sets.out["status"] & ~1).ne(0).sum().item())
+    value = world * N * args.steps / (ms * 1e-3)
+    # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
+    edits = float(2.0 * cnt[1] + 10.0)
+    abytes = algorithmic_bytes(cfg, edits, 0.0) * N
+    achieved = abytes / (ms * 1e-3 / args.steps) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "peak_kind": peak_kind, "traffic": None,
+                "algorithmic_bytes_per_launch": abytes, "kernel": "br_step_kernel<false,0>"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100..",
+                   "instances_per_launch": N, "rotating_sets": n_sets,
+                   "l2": f"{n_sets} instance sets stepped in rotation: data touched between two visits "
+                         f"of a set exceeds the 126 MB L2", "threads_per_instance": sets.router.params.threads},
+        "roofline": roofline, "clocks": clocks, "gpu_launches": args.steps,
+        "bad_status_instances": bad,
+    }
+
+    if rank == 0 and world == 1 and not args.quick:
+        # ---------------- end to end through the host-buffer entry point ----------------
+        line["e2e"] = e2e_host(torch, device, args)
+        # ---------------- extras: c4 batched BR-H, latency path ----------------
+        try:
+            line["extra"] = extras(torch, device, args, peak)
+        except Exception as ex:  # keep the headline line even if an extra fails
+            line["extra"] = {"error": repr(ex)}
+        # ---------------- CPU baseline: the checker on host cores ----------------
+        rate, done, dt = oracle_rate("c3", 12.0, 16, 500)
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"{done} instance-steps of c3 (16 instances), {dt:.1f} s, single thread"}
+    elif rank == 0:
+        line["e2e"] = None
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def e2e_host(torch, device, args):
+    from paper_2605_06113_b200.binding import Router
+    cfg = wlm.get_config("c3")
+    wl = wlm.make_workload(cfg, n_instances=cfg.N, first_instance=1 << 20)
+    r = Router(wl, device=device, threads=args.threads)
+    st = {k: torch.from_numpy(np.ascontiguousarray(v).view(
+        {np.dtype(np.uint64): np.int64, np.dtype(np.uint32): np.int32}.get(v.dtype, v.dtype))).pin_memory()
+          for k, v in wl.state.items()}
+    out = {k: v.pin_memory() for k, v in r.outputs(cfg.N, device="cpu").items()}
+    steps = 30
+    up = down = 0
+    for _ in range(3):
+        r.step_host(st, out)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        up, down = r.step_host(st, out)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    r.close()
+    return {"value": cfg.N * steps / dt, "unit": UNIT, "h2d_bytes_per_step": up,
+            "d2h_bytes_per_step": down, "steps": steps, "ms_per_step": 1e3 * dt / steps}
+
+
+def extras(torch, device, args, peak):
+    ex = {}
+    # c4: BR-H batched, term_probs ring of 8 step buffers (1 GiB) and 2 instance sets
+    cfg = wlm.get_config("c4")
+    sets = RotatingSets("c4", cfg.N, 2, device, seed_offset=0, probs_ring=4)
+    ms = time_launches(torch, sets.step, 20, 200)
+    cnt = sets.out["counters"].to(torch.float64).view(2, cfg.N, 4).mean(dim=(0, 1)).cpu().numpy()
+    abytes = algorithmic_bytes(cfg, float(2 * cnt[1] + 20), 1.0 / cfg.delta_T) * cfg.N
+    ach = abytes / (ms * 1e-3 / 200) / 1e9
+    ex["c4_batched"] = {"value": cfg.N * 200 / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / 200,
+                        "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                                     "frac": ach / peak, "algorithmic_bytes_per_launch": abytes}}
+    del sets
+    torch.cuda.empty_cache()
+    # c3 with 16 steps per launch (persistent multi-step form of the same kernel)
+    ex["latency"] = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
+                     latency_path(torch, "c4", device, 1000)]
+    return ex
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1920)
+    ap.add_argument("--warmup", type=int, default=80)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
+    ap.add_argument("--quick", action="store_true", help="headline measurement only")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        args.steps = min(args.steps, 400)
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

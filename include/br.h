@@ -1,0 +1,193 @@
+/*
+ * BalanceRoute routing step for data-parallel LLM decode, C ABI.
+ *
+ * One *routing instance* is a fleet of G decode workers with B request slots
+ * each plus a waiting set of prefill-completed requests (the cluster snapshot of
+ * Section 5, Eq. "cluster-snapshot").  br_step advances a batch of independent
+ * instances by one decode step k:
+ *
+ *   ARRIVE   new requests join R_wait(k) in arrival order      (Section 2.2)
+ *   PREDICT  c_hat maintenance and horizon projection (H > 0)   (Eqs. 3-6, Appendix "Refresh logic")
+ *   ROUTE    two-stage admission by F-score                     (Eq. 1 / Eq. 2, Algorithms 1 and 2)
+ *   RECORD   per-worker loads L_g(k) and (max, min, sum)        (Section 3.1, Section 5.1 "Metrics")
+ *   ADVANCE  every running request ends or grows by one token   (Section 2.2)
+ *
+ * All array arguments are DEVICE pointers owned by the caller unless a comment
+ * says "host".  The library keeps no pointer beyond a call, except those baked
+ * into a captured graph (br_graph_capture), which must stay valid until
+ * br_destroy.  Calls are asynchronous on the stream given in the batch and
+ * return a host status at once; nothing aborts, traps or prints.  A br_ctx must
+ * not be used from two host threads at the same time.
+ */
+#ifndef BR_H_
+#define BR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BR_VERSION 100
+
+/* status codes returned by every entry point */
+#define BR_OK        0
+#define BR_EINVAL   -1   /* null / misaligned pointer, or a size outside the limits below */
+#define BR_ERANGE   -2   /* a value range that the integer packing cannot represent       */
+#define BR_ECUDA    -3   /* a CUDA runtime call failed; br_strerror gives its text        */
+#define BR_ENOMEM   -4   /* host or device allocation failed (br_create, host-buffer path)*/
+#define BR_ESTATE   -5   /* call order violated (e.g. br_graph_step before capture)       */
+
+/* compiled limits */
+#define BR_MAX_G      64
+#define BR_MAX_H      16
+#define BR_MAX_B     256     /* B must be a multiple of 4                     */
+#define BR_MAX_W    4096     /* W must be a multiple of 4                     */
+#define BR_MAX_RMAX    5     /* Stage 2 enumerates 2^R_max - 1 <= 31 subsets   */
+
+#define BR_EMPTY_SLOT INT32_MIN  /* act_base value of a free slot              */
+
+/* per-instance status bits written to br_load_out.status */
+#define BR_ST_QUEUE_OVERFLOW  1u  /* at least one arrival was dropped (queue at W)   */
+#define BR_ST_ITER_CAP        2u  /* a routing loop hit its hard iteration bound     */
+#define BR_ST_BAD_STATE       4u  /* nact/occ/queue length inconsistent with limits  */
+
+typedef struct br_ctx br_ctx;
+
+/*
+ * Parameters, host memory, copied by br_create.  "default" = value used when the
+ * field is negative (or zero where zero is not meaningful).
+ */
+typedef struct {
+    int32_t B;              /* slots per worker (max concurrency B, Section 2.2)             */
+    int32_t W;              /* capacity of the waiting queue                                  */
+    int32_t R_max;          /* Stage-2 window (Algorithm 1); <= 0 -> 4                       */
+    int32_t S_greedy;       /* Stage-1 / Stage-2 threshold on total free slots; < 0 -> 2 G   */
+    double  alpha, beta, gamma; /* Eq. 2 parameters; ignored when score_mode == 0            */
+    int32_t delta_T;        /* c_hat refresh period; <= 0 -> max(1, H / 2)                   */
+    float   gate;           /* confidence gate on p_fin; < 0 -> 0.5                          */
+    float   c_floor;        /* lower bound of c_hat; < 0 -> 1                                */
+    int32_t score_mode;     /* 0: Eq. 1 in integers (needs H == 0); 1: Eq. 2 in fp64; < 0 -> 0 if H == 0 else 1 */
+    int32_t term_mode;      /* 0: requests never end; 1: end when Philox word < hazard_thr;
+                               2: end when 24-bit Philox uniform < term_probs[slot][0]       */
+    uint32_t hazard_thr;
+    const uint32_t *arr_cdf;/* device [rows][arr_len] Poisson CDF thresholds; the row for instance i
+                               at step k is i * arr_inst_stride + k % arr_period; NULL -> no arrivals */
+    int32_t arr_len, arr_period, arr_inst_stride;
+    const int32_t *len_tab; /* device [2^len_tab_log2] inverse-CDF table of prompt lengths   */
+    int32_t len_tab_log2;
+    int32_t burst_every, burst_size; /* burst_size extra arrivals when k > 0 and k % burst_every == 0 */
+    int32_t s_max;          /* largest prompt length the caller will ever enqueue (range proof) */
+    int32_t threads;        /* threads per instance (multiple of 32, <= 1024); <= 0 -> chosen from W and G*B */
+} br_params;
+
+/* running requests; instance i occupies row first_instance + i of every array */
+typedef struct {
+    int64_t  *load;       /* [N][G]   L_g at the start of the step (sum of cur over the worker)  */
+    int32_t  *nact;       /* [N][G]   |A_g|                                                     */
+    uint64_t *occ;        /* [N][G][ceil(B/64)] bit b set <=> slot b is occupied                */
+    int32_t  *act_base;   /* [N][G][B] cur - k of the request in the slot (constant while it
+                                       runs: cur = s_i + (k - x_i)), BR_EMPTY_SLOT if free      */
+    uint32_t *act_id;     /* [N][G][B] request id per slot; may be NULL                         */
+    float    *act_chat0;  /* [N][G][B] c_hat at the last refresh (H > 0 only, else may be NULL) */
+    uint8_t  *act_kref;   /* [N][G][B] step of the last refresh modulo 256 (H > 0 only)         */
+    int32_t  *step;       /* [N]      decode step k                                             */
+    uint64_t *seed;       /* [N]      Philox key of the instance                                */
+    uint32_t *next_id;    /* [N]      id given to the next arrival                              */
+} br_worker_state;
+
+/* waiting requests in arrival order; entries [n, W) are ignored */
+typedef struct {
+    int32_t  *s;          /* [N][W] prompt length s_i = w_i^(1)                                 */
+    uint32_t *id;         /* [N][W] request id                                                  */
+    int32_t  *n;          /* [N]    current length                                              */
+} br_waiting_queue;
+
+typedef struct {
+    int32_t n_instances;    /* instances in this call                                           */
+    int32_t first_instance; /* row offset into every per-instance array                         */
+    int32_t n_steps;        /* consecutive decode steps run by this one launch; <= 0 -> 1.  With
+                               n_steps > 1, term_probs, assign_out and every br_load_out array
+                               hold n_steps consecutive per-step blocks of n_instances rows,
+                               indexed from row 0 (first_instance must then be 0)              */
+    void   *stream;         /* cudaStream_t                                                     */
+} br_instance_batch;
+
+typedef struct {
+    int64_t  *load;       /* [N][G]  L_g(k) after this step's admissions                        */
+    int64_t  *trace;      /* [N][3]  (max_g L_g, min_g L_g, sum_g L_g); gives max-min, I(k), max/mean */
+    int32_t  *status;     /* [N]     BR_ST_* bits; may be NULL                                  */
+    uint32_t *counters;   /* [N][4]  this step: dropped arrivals, admissions, Stage-1 iterations,
+                                     Stage-2 pops; may be NULL                                  */
+    double   *fscore;     /* [N][W][G] optional: F_g({i}) of every waiting request before the
+                                     first admission (0 beyond the queue length); NULL in timed runs */
+} br_load_out;
+
+/*
+ * Creates a context for fleets of G workers and lookahead H (H = 0: BR-0).
+ * Validates sizes against the limits above and proves that loads and scores fit
+ * the 32-bit packings used on the device: B * (s_max + 2^22) < 2^31 (BR_ERANGE).
+ * Allocates only a small host object.  *out is set on BR_OK only.
+ */
+int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out);
+
+/*
+ * One decode step (or batch.n_steps of them) for batch.n_instances instances.
+ * Mutates worker_state and waiting_queue in place.
+ *   term_probs  [N][G][B][H] fp32 termination-classifier output for this step: entry h-1 is
+ *               the probability that the request ends at in-window step h given that it is
+ *               still running; NULL allowed when H == 0 and term_mode != 2
+ *   assign_out  [N][W] per queue position (as of after ARRIVE): g * B + slot of the admission,
+ *               -1 if the request keeps waiting or the position is beyond the queue
+ * Returns BR_EINVAL for null or misaligned (16-byte) array pointers and n_instances < 0,
+ * BR_ECUDA if the launch failed.  n_instances == 0 is a no-op returning BR_OK.
+ */
+int br_step(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
+            br_waiting_queue *waiting_queue, const float *term_probs, int32_t *assign_out,
+            br_load_out *load_out);
+
+/*
+ * Latency path: records one br_step launch with these arguments into a CUDA graph
+ * owned by ctx (replacing an earlier one); br_graph_step replays it on the stream
+ * given at capture.  The step counter lives in worker_state.step, so every replay
+ * advances by batch.n_steps steps; the caller refreshes term_probs in place.
+ */
+int br_graph_capture(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
+                     br_waiting_queue *waiting_queue, const float *term_probs,
+                     int32_t *assign_out, br_load_out *load_out);
+int br_graph_step(br_ctx *ctx);
+
+/*
+ * Host-buffer variant: every array pointer in worker_state, waiting_queue, term_probs,
+ * assign_out and load_out is a HOST pointer (pinned memory gives asynchronous copies).
+ * Copies the snapshot to device staging owned by ctx (grown on demand with cudaMalloc),
+ * runs the step, copies state and results back and synchronises the stream.
+ * h2d_bytes / d2h_bytes, if not NULL, receive the bytes moved in each direction.
+ * batch.n_steps must be 1 and batch.first_instance 0.
+ */
+int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
+                 br_waiting_queue *waiting_queue, const float *term_probs, int32_t *assign_out,
+                 br_load_out *load_out, int64_t *h2d_bytes, int64_t *d2h_bytes);
+
+/*
+ * F-score matrix alone (Eq. 1 / Eq. 2 for single requests): for n_requests prompt lengths s
+ * and per-instance projected loads Lh [N][G][H+1] (offset 0 = L_g(k)), writes
+ * F [N][n_requests][G] in fp64 and, if best_g is not NULL, argmax_g per request
+ * (lowest g on ties) restricted to workers with cap[g] > 0 (cap [N][G], may be NULL).
+ * This is the pool-bypass scorer of Appendix "Pool-bypass deployment path for BR-0"
+ * when H = 0 and Lh holds virtual loads.
+ */
+int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int32_t n_requests,
+              const int64_t *Lh, const int32_t *cap, double *F, int32_t *best_g);
+
+/* Frees the context, its staging buffers and graph.  NULL is accepted. */
+int br_destroy(br_ctx *ctx);
+
+/* Text for a status code; for BR_ECUDA the text of the last CUDA error seen by this library. */
+const char *br_strerror(int status);
+int br_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BR_H_ */

@@ -1,0 +1,338 @@
+// C-ABI entry points of the BalanceRoute routing library (declared in include/br.h).
+// Host side only validates, fills the kernel argument block and launches.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+
+#include "br_step.cuh"
+#include "br_fscore.cuh"
+
+using br::StepArgs;
+
+struct br_ctx {
+    int32_t G, H;
+    br_params p;              // resolved parameters
+    StepArgs base;            // constant part of the kernel arguments
+    int threads;
+    size_t smem;
+    // latency path
+    cudaGraph_t graph;
+    cudaGraphExec_t graph_exec;
+    cudaStream_t graph_stream;
+    // host-buffer path
+    void *stage;
+    size_t stage_bytes;
+};
+
+namespace {
+
+thread_local char g_cuda_msg[256] = "no CUDA error recorded";
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg), "%s: %s", what, cudaGetErrorString(e));
+    return BR_ECUDA;
+}
+#define BR_CUDA(call)                                      \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
+
+typedef void (*step_kernel_t)(const StepArgs);
+
+step_kernel_t pick_kernel(bool fp, int H)
+{
+    if (!fp) return br::br_step_kernel<false, 0>;
+    if (H == 0) return br::br_step_kernel<true, 0>;
+    if (H <= 4) return br::br_step_kernel<true, 4>;
+    if (H <= 8) return br::br_step_kernel<true, 8>;
+    return br::br_step_kernel<true, 16>;
+}
+
+int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_worker_state *ws,
+                    const br_waiting_queue *wq, const float *term_probs, const int32_t *assign_out,
+                    const br_load_out *out)
+{
+    if (!ctx || !b || !ws || !wq || !out) return BR_EINVAL;
+    if (b->n_instances < 0 || b->first_instance < 0) return BR_EINVAL;
+    const int n_steps = b->n_steps <= 0 ? 1 : b->n_steps;
+    if (n_steps > 1 && b->first_instance != 0) return BR_EINVAL;
+    if (!ws->load || !ws->nact || !ws->occ || !ws->act_base || !ws->step || !ws->seed || !ws->next_id)
+        return BR_EINVAL;
+    if (!wq->s || !wq->id || !wq->n) return BR_EINVAL;
+    if (!assign_out || !out->load || !out->trace) return BR_EINVAL;
+    if (ctx->H > 0 && (!ws->act_chat0 || !ws->act_kref || !term_probs)) return BR_EINVAL;
+    if (ctx->p.term_mode == 2 && !term_probs) return BR_EINVAL;
+    if (misaligned(ws->act_base, 16) || misaligned(wq->s, 16) || misaligned(wq->id, 16) ||
+        misaligned(assign_out, 16) || misaligned(ws->load, 8) || misaligned(ws->occ, 8) ||
+        misaligned(out->load, 8) || misaligned(out->trace, 8) || misaligned(ws->seed, 8) ||
+        (term_probs && misaligned(term_probs, 16)) || (out->fscore && misaligned(out->fscore, 8)))
+        return BR_EINVAL;
+    return BR_OK;
+}
+
+int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *ws,
+                const br_waiting_queue *wq, const float *term_probs, int32_t *assign_out,
+                const br_load_out *out, cudaStream_t stream)
+{
+    StepArgs a = ctx->base;
+    a.N = b->n_instances;
+    a.first_instance = b->first_instance;
+    a.n_steps = b->n_steps <= 0 ? 1 : b->n_steps;
+    a.ws = *ws;
+    a.wq = *wq;
+    a.term_probs = term_probs;
+    a.assign_out = assign_out;
+    a.out = *out;
+    step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H);
+    kern<<<b->n_instances, ctx->threads, ctx->smem, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
+    return BR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int br_version(void) { return BR_VERSION; }
+
+const char *br_strerror(int status)
+{
+    switch (status) {
+    case BR_OK: return "ok";
+    case BR_EINVAL: return "invalid argument (null or misaligned pointer, or size outside the compiled limits)";
+    case BR_ERANGE: return "value range too large for the device integer packing";
+    case BR_ECUDA: return g_cuda_msg;
+    case BR_ENOMEM: return "allocation failed";
+    case BR_ESTATE: return "call order violated";
+    default: return "unknown status";
+    }
+}
+
+int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
+{
+    if (!params || !out) return BR_EINVAL;
+    if (G < 1 || G > BR_MAX_G || H < 0 || H > BR_MAX_H) return BR_EINVAL;
+    br_params p = *params;
+    if (p.B < 4 || p.B > BR_MAX_B || (p.B % 4) != 0) return BR_EINVAL;
+    if (p.W < 4 || p.W > BR_MAX_W || (p.W % 4) != 0) return BR_EINVAL;
+    if (p.R_max <= 0) p.R_max = 4;
+    if (p.R_max > BR_MAX_RMAX) return BR_EINVAL;
+    if (p.S_greedy < 0) p.S_greedy = 2 * G;
+    if (p.delta_T <= 0) p.delta_T = H / 2 > 1 ? H / 2 : 1;
+    if (p.delta_T > 128) return BR_EINVAL;
+    if (p.gate < 0.0f) p.gate = 0.5f;
+    if (p.c_floor < 0.0f) p.c_floor = 1.0f;
+    if (p.score_mode < 0) p.score_mode = (H == 0) ? 0 : 1;
+    if (p.score_mode > 1 || (p.score_mode == 0 && H != 0)) return BR_EINVAL;
+    if (p.term_mode < 0 || p.term_mode > 2 || (p.term_mode == 2 && H == 0)) return BR_EINVAL;
+    if (p.arr_cdf) {
+        if (p.arr_len < 1 || p.arr_period < 1 || p.arr_inst_stride < 0 || !p.len_tab) return BR_EINVAL;
+        if (p.len_tab_log2 < 0 || p.len_tab_log2 > 24) return BR_EINVAL;
+        if (p.burst_every < 0 || p.burst_size < 0) return BR_EINVAL;
+    }
+    if (p.s_max <= 0) p.s_max = 1 << 20;
+    // loads and partial sums are carried in 32 bits on the device
+    if ((long long)p.B * ((long long)p.s_max + (1ll << 22)) >= (1ll << 31)) return BR_ERANGE;
+    if (p.score_mode == 1) {
+        if (!(p.alpha > 0.0) || !(p.gamma > 0.0) || !(p.gamma <= 1.0) || !(p.beta >= 0.0) ||
+            !isfinite(p.alpha) || !isfinite(p.beta))
+            return BR_EINVAL;
+    }
+    const int A = G * p.B;
+    if (p.threads > 0) {
+        if (p.threads % 32 != 0 || p.threads > 512) return BR_EINVAL;
+    } else {
+        int t = p.W / 8 > A / 16 ? p.W / 8 : A / 16;
+        t = (t + 31) / 32 * 32;
+        p.threads = t < 32 ? 32 : (t > 256 ? 256 : t);
+    }
+
+    br_ctx *ctx = new (std::nothrow) br_ctx();
+    if (!ctx) return BR_ENOMEM;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->G = G; ctx->H = H; ctx->p = p; ctx->threads = p.threads;
+    StepArgs &a = ctx->base;
+    a.G = G; a.H = H; a.B = p.B; a.W = p.W; a.R_max = p.R_max; a.S_greedy = p.S_greedy;
+    a.occ_words = (p.B + 63) / 64;
+    a.delta_T = p.delta_T; a.gate = p.gate; a.c_floor = p.c_floor;
+    a.term_mode = p.term_mode; a.hazard_thr = p.hazard_thr;
+    a.arr_cdf = p.arr_cdf; a.arr_len = p.arr_len; a.arr_period = p.arr_period;
+    a.arr_inst_stride = p.arr_inst_stride;
+    a.len_tab = p.len_tab; a.len_shift = 32 - p.len_tab_log2;
+    a.burst_every = p.burst_every; a.burst_size = p.burst_size;
+    // d = (1, gamma, ..., gamma^H) by repeated multiplication; D = 1^T d left to right
+    volatile double D = 0.0;
+    for (int h = 0; h <= BR_MAX_H; ++h) a.d[h] = 0.0;
+    if (p.score_mode == 1) {
+        for (int h = 0; h <= H; ++h) {
+            volatile double dh = (h == 0) ? 1.0 : a.d[h - 1] * p.gamma;
+            a.d[h] = dh;
+            D = D + dh;
+        }
+        volatile double aD = p.alpha * D;
+        a.aD = aD; a.beta = p.beta;
+    } else {
+        a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G;
+    }
+    ctx->smem = br::step_smem_bytes(G, H, p.W, a.occ_words);
+    *out = ctx;
+    return BR_OK;
+}
+
+int br_step(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *ws, br_waiting_queue *wq,
+            const float *term_probs, int32_t *assign_out, br_load_out *out)
+{
+    int rc = check_step_args(ctx, batch, ws, wq, term_probs, assign_out, out);
+    if (rc != BR_OK) return rc;
+    if (batch->n_instances == 0) return BR_OK;
+    return launch_step(ctx, batch, ws, wq, term_probs, assign_out, out, (cudaStream_t)batch->stream);
+}
+
+int br_graph_capture(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *ws,
+                     br_waiting_queue *wq, const float *term_probs, int32_t *assign_out,
+                     br_load_out *out)
+{
+    int rc = check_step_args(ctx, batch, ws, wq, term_probs, assign_out, out);
+    if (rc != BR_OK) return rc;
+    if (batch->n_instances == 0) return BR_EINVAL;
+    if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
+    if (ctx->graph) { cudaGraphDestroy(ctx->graph); ctx->graph = nullptr; }
+    cudaStream_t cap;
+    BR_CUDA(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
+    cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) { cudaStreamDestroy(cap); return cuda_fail(e, "cudaStreamBeginCapture"); }
+    rc = launch_step(ctx, batch, ws, wq, term_probs, assign_out, out, cap);
+    e = cudaStreamEndCapture(cap, &ctx->graph);
+    cudaStreamDestroy(cap);
+    if (rc != BR_OK) return rc;
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamEndCapture");
+    BR_CUDA(cudaGraphInstantiate(&ctx->graph_exec, ctx->graph, 0));
+    ctx->graph_stream = (cudaStream_t)batch->stream;
+    return BR_OK;
+}
+
+int br_graph_step(br_ctx *ctx)
+{
+    if (!ctx) return BR_EINVAL;
+    if (!ctx->graph_exec) return BR_ESTATE;
+    BR_CUDA(cudaGraphLaunch(ctx->graph_exec, ctx->graph_stream));
+    return BR_OK;
+}
+
+int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *hws,
+                 br_waiting_queue *hwq, const float *h_probs, int32_t *h_assign, br_load_out *hout,
+                 int64_t *h2d_bytes, int64_t *d2h_bytes)
+{
+    if (!ctx || !batch || !hws || !hwq || !hout) return BR_EINVAL;
+    if (batch->n_instances < 0 || batch->first_instance != 0 || batch->n_steps > 1) return BR_EINVAL;
+    if (!hws->load || !hws->nact || !hws->occ || !hws->act_base || !hws->step || !hws->seed ||
+        !hws->next_id || !hwq->s || !hwq->id || !hwq->n || !h_assign || !hout->load || !hout->trace)
+        return BR_EINVAL;
+    if (ctx->H > 0 && (!hws->act_chat0 || !hws->act_kref || !h_probs)) return BR_EINVAL;
+    if (ctx->p.term_mode == 2 && !h_probs) return BR_EINVAL;
+    const size_t N = (size_t)batch->n_instances;
+    if (N == 0) return BR_OK;
+    const size_t G = ctx->G, H = ctx->H, B = ctx->p.B, W = ctx->p.W, A = G * B;
+    const size_t OW = (B + 63) / 64;
+    cudaStream_t st = (cudaStream_t)batch->stream;
+
+    // staging layout: every block padded to 256 bytes
+    struct Blk { size_t bytes; void **dev; void *host; bool in, out; };
+    br_worker_state dws; memset(&dws, 0, sizeof(dws));
+    br_waiting_queue dwq; memset(&dwq, 0, sizeof(dwq));
+    br_load_out dout; memset(&dout, 0, sizeof(dout));
+    float *d_probs = nullptr; int32_t *d_assign = nullptr;
+    const bool pred = H > 0;
+    Blk blks[] = {
+        {N * G * 8, (void **)&dws.load, hws->load, true, true},
+        {N * G * 4, (void **)&dws.nact, hws->nact, true, true},
+        {N * G * OW * 8, (void **)&dws.occ, hws->occ, true, true},
+        {N * A * 4, (void **)&dws.act_base, hws->act_base, true, true},
+        {hws->act_id ? N * A * 4 : 0, (void **)&dws.act_id, hws->act_id, true, true},
+        {pred ? N * A * 4 : 0, (void **)&dws.act_chat0, hws->act_chat0, true, true},
+        {pred ? N * A : 0, (void **)&dws.act_kref, hws->act_kref, true, true},
+        {N * 4, (void **)&dws.step, hws->step, true, true},
+        {N * 8, (void **)&dws.seed, hws->seed, true, false},
+        {N * 4, (void **)&dws.next_id, hws->next_id, true, true},
+        {N * W * 4, (void **)&dwq.s, hwq->s, true, true},
+        {N * W * 4, (void **)&dwq.id, hwq->id, true, true},
+        {N * 4, (void **)&dwq.n, hwq->n, true, true},
+        {h_probs ? N * A * H * 4 : 0, (void **)&d_probs, (void *)h_probs, true, false},
+        {N * W * 4, (void **)&d_assign, h_assign, false, true},
+        {N * G * 8, (void **)&dout.load, hout->load, false, true},
+        {N * 3 * 8, (void **)&dout.trace, hout->trace, false, true},
+        {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
+        {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
+        {hout->fscore ? N * W * G * 8 : 0, (void **)&dout.fscore, hout->fscore, false, true},
+    };
+    size_t total = 0;
+    for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;
+    if (total > ctx->stage_bytes) {
+        if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+        cudaError_t e = cudaMalloc(&ctx->stage, total);
+        if (e != cudaSuccess) { cuda_fail(e, "cudaMalloc(staging)"); return BR_ENOMEM; }
+        ctx->stage_bytes = total;
+    }
+    size_t off = 0; int64_t up = 0, down = 0;
+    for (Blk &b : blks) {
+        if (!b.bytes) continue;
+        *b.dev = (char *)ctx->stage + off;
+        off += (b.bytes + 255) & ~(size_t)255;
+        if (b.in) { BR_CUDA(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, st)); up += (int64_t)b.bytes; }
+    }
+    br_instance_batch db = *batch; db.n_steps = 1;
+    int rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
+    if (rc != BR_OK) return rc;
+    rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
+    if (rc != BR_OK) return rc;
+    for (Blk &b : blks) {
+        if (!b.bytes || !b.out) continue;
+        BR_CUDA(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, st));
+        down += (int64_t)b.bytes;
+    }
+    BR_CUDA(cudaStreamSynchronize(st));
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return BR_OK;
+}
+
+int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int32_t n_requests,
+              const int64_t *Lh, const int32_t *cap, double *F, int32_t *best_g)
+{
+    if (!ctx || !batch || !s || !Lh || !F) return BR_EINVAL;
+    if (batch->n_instances < 0 || n_requests < 0 || (n_requests % 4) != 0) return BR_EINVAL;
+    if (misaligned(s, 16) || misaligned(Lh, 8) || misaligned(F, 8)) return BR_EINVAL;
+    if (batch->n_instances == 0 || n_requests == 0) return BR_OK;
+    br::FscoreArgs a;
+    a.G = ctx->G; a.H = ctx->H; a.fp = ctx->p.score_mode == 1;
+    a.aD = ctx->base.aD; a.beta = ctx->base.beta;
+    for (int h = 0; h <= BR_MAX_H; ++h) a.d[h] = ctx->base.d[h];
+    a.n_req = n_requests; a.first_instance = batch->first_instance;
+    a.s = s; a.Lh = Lh; a.cap = cap; a.F = F; a.best_g = best_g;
+    const int tiles = (n_requests + br::kFsTile - 1) / br::kFsTile;
+    dim3 grid(tiles, batch->n_instances);
+    br::br_fscore_kernel<<<grid, 256, 0, (cudaStream_t)batch->stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "br_fscore launch");
+    return BR_OK;
+}
+
+int br_destroy(br_ctx *ctx)
+{
+    if (!ctx) return BR_OK;
+    if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
+    if (ctx->graph) cudaGraphDestroy(ctx->graph);
+    if (ctx->stage) cudaFree(ctx->stage);
+    delete ctx;
+    return BR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,97 @@
+"""CUDA library against the CPU checker, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2605_06113_b200 import workload as wlm
+from helpers import run_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c0_br0_full_run():
+    run_parity(wlm.get_config("c0"), 1, 300, check_every=10, fscore=True)
+
+
+@pytest.mark.parametrize("threads", [32, 64, 256])
+def test_c1_br0_thread_shapes(threads):
+    run_parity(wlm.get_config("c1"), 1, 150, threads=threads, check_every=25)
+
+
+def test_c1_br0_full_run():
+    run_parity(wlm.get_config("c1"), 1, 2000, check_every=100)
+
+
+def test_c2_brh_full_run():
+    run_parity(wlm.get_config("c2"), 1, 2000, check_every=100)
+
+
+def test_c2_brh_fscore_matrix():
+    run_parity(wlm.get_config("c2"), 1, 60, check_every=10, fscore=True)
+
+
+def test_c2_brh_open_gate_every_step():
+    # the probability path exercised at scale: gate open for everyone, refresh every step
+    run_parity(wlm.get_config("c2", gate=0.0, delta_T=1), 2, 300, check_every=20)
+
+
+def test_c2_brh_low_gate_period_two():
+    run_parity(wlm.get_config("c2", gate=0.12, delta_T=2, beta=43.0, gamma=0.86), 2, 300, check_every=20)
+
+
+def test_c3_br0_batched_slice():
+    run_parity(wlm.get_config("c3"), 6, 200, check_every=20)
+
+
+def test_c4_brh_batched_slice():
+    run_parity(wlm.get_config("c4"), 3, 260, check_every=20)
+
+
+def test_c4_brh_hazard_informative_probs():
+    # classifier output that is confident for some requests: gate opens request by request
+    run_parity(wlm.get_config("c4", beta_ab=(0.5, 2.0), gate=0.5, term_mode=2), 2, 80, check_every=10)
+
+
+@pytest.mark.parametrize("S_greedy", [0, 16, 1 << 20])
+def test_stage_split_sweep(S_greedy):
+    # 0: Stage 1 admits everything; huge: Stage 2 only
+    run_parity(wlm.get_config("c1", S_greedy=S_greedy), 1, 120, check_every=20)
+
+
+@pytest.mark.parametrize("R_max", [1, 2, 5])
+def test_window_sizes(R_max):
+    run_parity(wlm.get_config("c1", R_max=R_max), 1, 120, check_every=20)
+
+
+def test_brh_code_path_at_h0_matches_br0():
+    cfg = wlm.get_config("c1")
+    a = run_parity(cfg, 1, 200, check_every=50)
+    b = run_parity(wlm.get_config("c1", score_mode=1, alpha=1.0, beta=float(cfg.G), gamma=0.64), 1, 200,
+                   check_every=50)
+    assert np.array_equal(a, b)
+
+
+def test_multi_step_launch_and_graph_replay():
+    run_parity(wlm.get_config("c1"), 2, 120, launch_steps=8, check_every=1)
+    run_parity(wlm.get_config("c2"), 1, 96, launch_steps=4, check_every=1)
+    run_parity(wlm.get_config("c1"), 1, 100, graph=True, check_every=10)
+    run_parity(wlm.get_config("c2"), 1, 100, graph=True, check_every=10)
+
+
+def test_ragged_shapes():
+    # G not a multiple of anything, B = 12 (not a multiple of 32), tiny and odd queue capacities
+    for G, B, W, H in [(1, 4, 4, 0), (3, 12, 20, 0), (5, 12, 36, 3), (7, 36, 100, 2), (64, 8, 64, 16)]:
+        cfg = wlm.get_config("c0", G=G, B=B, W=W, H=H, init_active=B // 2, init_queue=W // 2,
+                             hazard=0.05, term_mode=1, arrival=("const", 3.0), S_greedy=-1,
+                             score_mode=-1, delta_T=-1, gate=0.1)
+        run_parity(cfg, 3, 80, check_every=10)
+
+
+def test_empty_and_saturated_edges():
+    # nothing waiting and nothing arriving; then full workers with a full queue and no terminations
+    cfg = wlm.get_config("c0", init_queue=0, arrival=("const", 1e-9))
+    run_parity(cfg, 1, 20)
+    cfg = wlm.get_config("c1", term_mode=0, hazard=0.0)
+    run_parity(cfg, 1, 20)
+    # empty fleet, long queue: first step admits min(S_tot, n_w)
+    cfg = wlm.get_config("c1", init_active=0)
+    run_parity(cfg, 1, 10)
