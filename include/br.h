@@ -78,7 +78,7 @@ typedef struct {
     int32_t len_tab_log2;
     int32_t burst_every, burst_size; /* burst_size extra arrivals when k > 0 and k % burst_every == 0 */
     int32_t s_max;          /* largest prompt length the caller will ever enqueue (range proof) */
-    int32_t threads;        /* threads per instance (multiple of 32, <= 1024); <= 0 -> chosen from W and G*B */
+    int32_t threads;        /* threads per instance (multiple of 32, <= 256); <= 0 -> chosen from G*B, H and the batch size */
 } br_params;
 
 /* running requests; instance i occupies row first_instance + i of every array */
@@ -121,12 +121,18 @@ typedef struct {
                                      Stage-2 pops; may be NULL                                  */
     double   *fscore;     /* [N][W][G] optional: F_g({i}) of every waiting request before the
                                      first admission (0 beyond the queue length); NULL in timed runs */
+    uint32_t *phase_cycles; /* [N][6] optional: SM clock cycles this step spent in ARRIVE, PREDICT,
+                                     Stage 1, Stage 2, RECORD + queue compaction, ADVANCE (the split the
+                                     paper reports for its dispatcher: preparation / Stage 1 / Stage 2);
+                                     may be NULL */
 } br_load_out;
 
 /*
  * Creates a context for fleets of G workers and lookahead H (H = 0: BR-0).
- * Validates sizes against the limits above and proves that loads and scores fit
- * the 32-bit packings used on the device: B * (s_max + 2^22) < 2^31 (BR_ERANGE).
+ * Validates sizes against the limits above and proves that queue keys, loads and
+ * Eq. 1 scores fit the 32-bit arithmetic used on the device (else BR_ERANGE):
+ * s_max * 2^ceil(log2 W) < 2^31, B * (s_max + 2^22) < 2^31 (a request may run for at
+ * most 2^22 steps), G * R_max * s_max < 2^31.  Prompt lengths must be >= 1.
  * Allocates only a small host object.  *out is set on BR_OK only.
  */
 int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out);

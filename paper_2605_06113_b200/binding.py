@@ -48,7 +48,8 @@ class BrInstanceBatch(C.Structure):
 
 
 class BrLoadOut(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("load", "trace", "status", "counters", "fscore")]
+    _fields_ = [(n, C.c_void_p) for n in ("load", "trace", "status", "counters", "fscore",
+                                          "phase_cycles")]
 
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
@@ -182,7 +183,8 @@ class Router:
                                "step", "seed", "next_id")})
         wq = BrWaitingQueue(s=_ptr(st["wq_s"]), id=_ptr(st["wq_id"]), n=_ptr(st["wq_n"]))
         lo = BrLoadOut(load=_ptr(out["load"]), trace=_ptr(out["trace"]), status=_ptr(out.get("status")),
-                       counters=_ptr(out.get("counters")), fscore=_ptr(out.get("fscore")))
+                       counters=_ptr(out.get("counters")), fscore=_ptr(out.get("fscore")),
+                       phase_cycles=_ptr(out.get("phase_cycles")))
         b = BrInstanceBatch(n_instances=N, first_instance=first, n_steps=n_steps, stream=stream)
         return b, ws, wq, lo
 

@@ -16,7 +16,8 @@ struct br_ctx {
     int32_t G, H;
     br_params p;              // resolved parameters
     StepArgs base;            // constant part of the kernel arguments
-    int threads;
+    int threads;              // threads per instance for large batches
+    int threads_small;        // ... for batches of a few instances (latency path)
     size_t smem;
     // latency path
     cudaGraph_t graph;
@@ -46,13 +47,19 @@ inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintp
 
 typedef void (*step_kernel_t)(const StepArgs);
 
-step_kernel_t pick_kernel(bool fp, int H)
+template <int GW>
+step_kernel_t pick_kernel_gw(bool fp, int H)
 {
-    if (!fp) return br::br_step_kernel<false, 0>;
-    if (H == 0) return br::br_step_kernel<true, 0>;
-    if (H <= 4) return br::br_step_kernel<true, 4>;
-    if (H <= 8) return br::br_step_kernel<true, 8>;
-    return br::br_step_kernel<true, 16>;
+    if (!fp) return br::br_step_kernel<false, 0, GW>;
+    if (H == 0) return br::br_step_kernel<true, 0, GW>;
+    if (H <= 4) return br::br_step_kernel<true, 4, GW>;
+    if (H <= 8) return br::br_step_kernel<true, 8, GW>;
+    return br::br_step_kernel<true, 16, GW>;
+}
+
+step_kernel_t pick_kernel(bool fp, int H, int G)
+{
+    return G <= 32 ? pick_kernel_gw<1>(fp, H) : pick_kernel_gw<2>(fp, H);
 }
 
 int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_worker_state *ws,
@@ -90,8 +97,10 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.term_probs = term_probs;
     a.assign_out = assign_out;
     a.out = *out;
-    step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H);
-    kern<<<b->n_instances, ctx->threads, ctx->smem, stream>>>(a);
+    step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G);
+    // few instances: the launch is latency-bound, so spread each instance over more warps
+    const int threads = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
+    kern<<<b->n_instances, threads, ctx->smem, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
     return BR_OK;
@@ -138,30 +147,43 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         if (p.len_tab_log2 < 0 || p.len_tab_log2 > 24) return BR_EINVAL;
         if (p.burst_every < 0 || p.burst_size < 0) return BR_EINVAL;
     }
-    if (p.s_max <= 0) p.s_max = 1 << 20;
-    // loads and partial sums are carried in 32 bits on the device
+    int wl = 2;
+    while ((1 << wl) < p.W) ++wl;
+    if (p.s_max <= 0) p.s_max = (1 << (31 - wl)) - 1 < (1 << 20) ? (1 << (31 - wl)) - 1 : (1 << 20);
+    // range proofs for the 32-bit device arithmetic:
+    //   packed queue keys  s * 2^wl + position        < 2^31
+    //   loads and partial sums  B * (s_max + 2^22)     < 2^31   (requests older than 2^22 steps are not supported)
+    //   Eq. 1 scores  G * R_max * s_max                < 2^31
+    if ((long long)p.s_max >= (1ll << (31 - wl))) return BR_ERANGE;
     if ((long long)p.B * ((long long)p.s_max + (1ll << 22)) >= (1ll << 31)) return BR_ERANGE;
+    if ((long long)G * p.R_max * (long long)p.s_max >= (1ll << 31)) return BR_ERANGE;
     if (p.score_mode == 1) {
         if (!(p.alpha > 0.0) || !(p.gamma > 0.0) || !(p.gamma <= 1.0) || !(p.beta >= 0.0) ||
             !isfinite(p.alpha) || !isfinite(p.beta))
             return BR_EINVAL;
     }
     const int A = G * p.B;
+    int threads_small, threads_large;
     if (p.threads > 0) {
-        if (p.threads % 32 != 0 || p.threads > 512) return BR_EINVAL;
+        if (p.threads % 32 != 0 || p.threads > 256) return BR_EINVAL;
+        threads_small = threads_large = p.threads;
     } else {
-        int t = p.W / 8 > A / 16 ? p.W / 8 : A / 16;
-        t = (t + 31) / 32 * 32;
-        p.threads = t < 32 ? 32 : (t > 256 ? 256 : t);
+        const int work = A * (H > 0 ? 2 : 1);
+        int w = (work + 2047) / 2048;
+        threads_large = 32 * (w < 1 ? 1 : (w > 8 ? 8 : w));
+        w = (work + 1023) / 1024;
+        threads_small = 32 * (w < 1 ? 1 : (w > 8 ? 8 : w));
     }
 
     br_ctx *ctx = new (std::nothrow) br_ctx();
     if (!ctx) return BR_ENOMEM;
     memset(ctx, 0, sizeof(*ctx));
-    ctx->G = G; ctx->H = H; ctx->p = p; ctx->threads = p.threads;
+    ctx->G = G; ctx->H = H; ctx->p = p;
+    ctx->threads = threads_large; ctx->threads_small = threads_small;
     StepArgs &a = ctx->base;
     a.G = G; a.H = H; a.B = p.B; a.W = p.W; a.R_max = p.R_max; a.S_greedy = p.S_greedy;
     a.occ_words = (p.B + 63) / 64;
+    a.wl = wl;
     a.delta_T = p.delta_T; a.gate = p.gate; a.c_floor = p.c_floor;
     a.term_mode = p.term_mode; a.hazard_thr = p.hazard_thr;
     a.arr_cdf = p.arr_cdf; a.arr_len = p.arr_len; a.arr_period = p.arr_period;
@@ -182,7 +204,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     } else {
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G;
     }
-    ctx->smem = br::step_smem_bytes(G, H, p.W, a.occ_words);
+    ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
     *out = ctx;
     return BR_OK;
 }
@@ -272,6 +294,7 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
         {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
         {hout->fscore ? N * W * G * 8 : 0, (void **)&dout.fscore, hout->fscore, false, true},
+        {hout->phase_cycles ? N * 24 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
     };
     size_t total = 0;
     for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;

@@ -2,9 +2,15 @@
 //
 // Phases per decode step k (Section 2.2 model; Algorithms 1 and 2):
 //   ARRIVE -> PREDICT (H > 0) -> ROUTE (Stage 1, Stage 2) -> RECORD -> ADVANCE.
-// Worker-level state (loads, projected loads, envelope, free slots) lives in shared
-// memory; the waiting queue is staged in shared memory with coalesced 16-byte loads;
-// every arg-max is a warp-shuffle reduction with a lowest-index tie-break.
+//
+// Warp 0 is the router.  It keeps the per-worker state (free slots, projected loads
+// L_g(k+h), envelope M_h) in registers, one or two workers per lane, and walks the
+// sequential admission loop with warp reductions only: no block barrier sits on the
+// admission chain.  The waiting queue lives in shared memory as packed 32-bit keys
+// (prompt length in the high bits, inverted position in the low bits) so that "largest
+// s, earliest arrival" is one integer max.  All warps stream the running-request state
+// (PREDICT, ADVANCE) with coalesced 16-byte loads issued in batches; while warp 0 routes,
+// the other warps already draw the Philox termination words of the step.
 #pragma once
 #include "br_device.cuh"
 #include "../../include/br.h"
@@ -13,6 +19,7 @@ namespace br {
 
 struct StepArgs {
     int32_t G, H, B, W, R_max, S_greedy, occ_words;
+    int32_t wl;                 // log2 of the queue-position field of a packed key
     int32_t delta_T;
     float gate, c_floor;
     int32_t term_mode;
@@ -33,86 +40,38 @@ struct StepArgs {
 };
 
 // shared-memory footprint of one instance (bytes), mirrored by the host
-__host__ __device__ inline size_t step_smem_bytes(int G, int H, int W, int occ_words)
+__host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words)
 {
     size_t n = 0;
-    n += sizeof(long long) * (size_t)G * (H + 1);   // Lh
-    n += sizeof(long long) * (size_t)(H + 1);       // Mh
-    n += sizeof(long long) * (size_t)G;             // load_new
-    n += sizeof(unsigned long long) * (size_t)G * occ_words;
-    n += sizeof(long long) * 64;                    // red_key
-    n += sizeof(int) * 64 * 2;                      // red_idx, red_val
-    n += sizeof(int) * (size_t)W * 2;               // q_s, q_id
-    n += sizeof(int) * (size_t)G * 2;               // cap, nact_new
-    n += sizeof(int) * 8;                           // scalars
+    n += 4 * (size_t)W;                          // q_key
+    n += 8 * (size_t)G * occ_words;              // occ
+    n += 4 * (size_t)G * (H + 1);                // Lh_s (PREDICT accumulators)
+    n += 4 * (size_t)G * 2;                      // load_new, nact_new
+    n += ((size_t)G * B / 4 + 15) & ~(size_t)15; // term_nib
+    n += 64;                                     // scalars
     return (n + 15) & ~(size_t)15;
 }
 
-struct BestV {
-    long long key;
-    int idx;
-    int val;
-};
-
-// block arg-max carrying a 32-bit payload of the winner
-__device__ __forceinline__ BestV block_argmax_v(long long key, int idx, int val, long long *red_key,
-                                                int *red_idx, int *red_val, int &phase)
-{
-    Best b{key, idx};
-    Best w = warp_argmax(b);
-    const unsigned src = __ballot_sync(kFull, idx == w.idx && key == w.key);
-    int v = __shfl_sync(kFull, val, src ? (__ffs(src) - 1) : 0);
-    const int nwarps = blockDim.x >> 5;
-    if (nwarps == 1) return BestV{w.key, w.idx, v};
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    long long *rk = red_key + phase * 32;
-    int *ri = red_idx + phase * 32;
-    int *rv = red_val + phase * 32;
-    phase ^= 1;
-    if (lane == 0) { rk[warp] = w.key; ri[warp] = w.idx; rv[warp] = v; }
-    __syncthreads();
-    Best c;
-    c.key = lane < nwarps ? rk[lane] : kNoKey;
-    c.idx = lane < nwarps ? ri[lane] : kNoIdx;
-    const int cv = lane < nwarps ? rv[lane] : 0;
-    Best w2 = warp_argmax(c);
-    const unsigned src2 = __ballot_sync(kFull, c.idx == w2.idx && c.key == w2.key);
-    const int v2 = __shfl_sync(kFull, cv, src2 ? (__ffs(src2) - 1) : 0);
-    return BestV{w2.key, w2.idx, v2};
-}
-
-// Score of admitting total prompt length `delta` to the worker whose margins were
-// loaded: Eq. 1 in int64 (FP = false) or Eq. 2 in fp64, term by term in h (FP = true).
-// Returned as an order- and sign-preserving int64 key.
+// Order- and sign-preserving key of a score: Eq. 1 in integers (FP = false) or Eq. 2 in
+// fp64 evaluated term by term in h (FP = true).
 template <bool FP, int HM>
 struct Scorer {
-    long long mi;
-    double md[HM + 1];
+    int mi;                 // Eq. 1 margin
+    double md[HM + 1];      // Eq. 2 margins
 
-    __device__ __forceinline__ void load(const long long *Lh, const long long *Mh, int g, int H)
-    {
-        const int H1 = H + 1;
-        if (!FP) {
-            mi = Mh[0] - Lh[g * H1];
-        } else {
-#pragma unroll
-            for (int h = 0; h <= HM; ++h)
-                md[h] = (h <= H) ? (double)(Mh[h] - Lh[g * H1 + h]) : 0.0;
-        }
-    }
     __device__ __forceinline__ long long key(const StepArgs &a, int delta) const
     {
         if (!FP) {
-            long long over = (long long)delta - mi;
+            int over = delta - mi;
             over = over > 0 ? over : 0;
-            return (long long)delta - (long long)a.G * over;
+            return (long long)(delta - a.G * over);        // |F| < 2^31 by the create-time proof
         } else {
             const double dl = (double)delta;
             double pen = 0.0;
 #pragma unroll
             for (int h = 0; h <= HM; ++h) {
                 if (h <= a.H) {
-                    double over = __dsub_rn(dl, md[h]);          // exact: integers below 2^53
+                    double over = __dsub_rn(dl, md[h]);     // exact: integers below 2^53
                     over = over > 0.0 ? over : 0.0;
                     pen = __dadd_rn(pen, __dmul_rn(a.d[h], over));
                 }
@@ -120,36 +79,50 @@ struct Scorer {
             return key_of_double(__dsub_rn(__dmul_rn(a.aD, dl), __dmul_rn(a.beta, pen)));
         }
     }
-    __device__ __forceinline__ double value(long long k) const
+    __device__ __forceinline__ static double value(long long k)
     {
         return FP ? double_of_key(k) : (double)k;
     }
 };
 
-template <bool FP, int HM>
-__global__ void __launch_bounds__(512) br_step_kernel(const StepArgs a)
+// warp arg-max of (64-bit key, then largest 32-bit tie value); returns the winning lane
+__device__ __forceinline__ int warp_argmax_lane(long long key, unsigned tie, long long &wkey)
+{
+    const int hi = (int)(key >> 32);
+    const unsigned lo = (unsigned)key;
+    const int mhi = __reduce_max_sync(kFull, hi);
+    const bool in1 = hi == mhi;
+    const unsigned mlo = __reduce_max_sync(kFull, in1 ? lo : 0u);
+    const bool in2 = in1 && lo == mlo;
+    const unsigned mt = __reduce_max_sync(kFull, in2 ? tie : 0u);
+    const unsigned who = __ballot_sync(kFull, in2 && tie == mt);
+    wkey = (long long)(((unsigned long long)(unsigned)mhi << 32) | mlo);
+    return __ffs(who) - 1;
+}
+
+constexpr int kUnroll = 4;      // 16-byte loads in flight per thread in the streaming phases
+
+template <bool FP, int HM, int GW>
+__global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31;
+    const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int nwarps = NT >> 5;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
+    const int WL = a.wl;
+    const unsigned posmask = (1u << WL) - 1u;
     const int inst = a.first_instance + blockIdx.x;
 
     // ---- shared-memory carve-up (sizes match step_smem_bytes) ----
-    int *q_s = reinterpret_cast<int *>(smem_raw);                     // 16-byte aligned
-    unsigned *q_id = reinterpret_cast<unsigned *>(q_s + W);          // W % 4 == 0
-    long long *Lh = reinterpret_cast<long long *>(q_id + W);
-    long long *Mh = Lh + (size_t)G * H1;
-    long long *load_new = Mh + H1;
-    unsigned long long *occ = reinterpret_cast<unsigned long long *>(load_new + G);
-    long long *red_key = reinterpret_cast<long long *>(occ + (size_t)G * OW);
-    int *red_idx = reinterpret_cast<int *>(red_key + 64);
-    int *red_val = red_idx + 64;
-    int *cap = red_val + 64;
-    int *nact_new = cap + G;
-    int *scal = nact_new + G;   // [0] admitted [1] Stage-1 iterations [2] Stage-2 pops [3],[4] status bits
-    int phase = 0;
-    if (tid < 8) scal[tid] = 0;
-    __syncthreads();
+    int *q_key = reinterpret_cast<int *>(smem_raw);                                 // [W]
+    unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_key + W);    // [G][OW]
+    unsigned *Lh_s = reinterpret_cast<unsigned *>(occ + (size_t)G * OW);            // [G][H1]
+    unsigned *load_new = Lh_s + (size_t)G * H1;                                     // [G]
+    int *nact_new = reinterpret_cast<int *>(load_new + G);                          // [G]
+    unsigned char *term_nib = reinterpret_cast<unsigned char *>(nact_new + G);      // [A/4]
+    int *scal = reinterpret_cast<int *>(term_nib + (((size_t)A / 4 + 15) & ~(size_t)15));
+    // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
+    //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue
 
     // ---- per-instance global rows ----
     long long *g_load = reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G;
@@ -167,30 +140,52 @@ __global__ void __launch_bounds__(512) br_step_kernel(const StepArgs a)
     int k = a.ws.step[inst];
     uint32_t next_id = a.ws.next_id[inst];
     int n_w = a.wq.n[inst];
-    int status = 0;
-    if (n_w < 0 || n_w > W) { status |= BR_ST_BAD_STATE; n_w = n_w < 0 ? 0 : W; }   // uniform
+    int prologue_status = 0;
+    if (n_w < 0 || n_w > W) { prologue_status |= BR_ST_BAD_STATE; n_w = n_w < 0 ? 0 : W; }
 
-    // queue -> shared memory (16-byte loads)
+    if (tid < 16) scal[tid] = 0;
+    // queue -> packed keys in shared memory (16-byte loads)
     for (int i = tid * 4; i < n_w; i += NT * 4) {
         const int4 v = *reinterpret_cast<const int4 *>(g_qs + i);
-        const uint4 u = *reinterpret_cast<const uint4 *>(g_qid + i);
-        *reinterpret_cast<int4 *>(q_s + i) = v;
-        *reinterpret_cast<uint4 *>(q_id + i) = u;
-    }
-    for (int g = tid; g < G; g += NT) {
-        int na = g_nact[g];
-        if (na < 0 || na > B) { atomicOr(&scal[4], (int)BR_ST_BAD_STATE); na = na < 0 ? 0 : B; }
-        cap[g] = B - na;
-        if (H == 0) Lh[g] = g_load[g];
+        int4 kk;
+        kk.x = (v.x << WL) | (int)(posmask - (unsigned)(i + 0));
+        kk.y = (v.y << WL) | (int)(posmask - (unsigned)(i + 1));
+        kk.z = (v.z << WL) | (int)(posmask - (unsigned)(i + 2));
+        kk.w = (v.w << WL) | (int)(posmask - (unsigned)(i + 3));
+        *reinterpret_cast<int4 *>(q_key + i) = kk;
     }
     for (int i = tid; i < G * OW; i += NT) occ[i] = g_occ[i];
+    for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
+    for (int i = tid; i < G; i += NT) { load_new[i] = 0u; nact_new[i] = 0; }
+
+    // router registers: lane owns workers lane and lane + 32
+    int cap[GW];
+    int L[GW][HM + 1];
+    int Mh[HM + 1];
+#pragma unroll
+    for (int h = 0; h <= HM; ++h) Mh[h] = 0;
+#pragma unroll
+    for (int w = 0; w < GW; ++w) {
+        const int g = lane + 32 * w;
+        cap[w] = -1;
+#pragma unroll
+        for (int h = 0; h <= HM; ++h) L[w][h] = 0;
+        if (warp == 0 && g < G) {
+            int na = g_nact[g];
+            if (na < 0 || na > B) { prologue_status |= BR_ST_BAD_STATE; na = na < 0 ? 0 : B; }
+            cap[w] = B - na;
+            L[w][0] = (int)g_load[g];
+        }
+    }
+    __syncthreads();
+    if (prologue_status) atomicOr(&scal[5], prologue_status);
 
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + inst;
         const float *probs = a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr;
-        int32_t *assign = a.assign_out + orow * W;
-        if (tid < 4) scal[tid] = 0;
-        if (H > 0) for (int i = tid; i < G * H1; i += NT) Lh[i] = 0;
+        long long t_phase[7];
+        const bool timing = a.out.phase_cycles != nullptr && tid == 0;
+        if (timing) t_phase[0] = clock64();
 
         // ================= ARRIVE =================
         int n_arr = 0;
@@ -205,360 +200,492 @@ __global__ void __launch_bounds__(512) br_step_kernel(const StepArgs a)
             }
             if (a.burst_every > 0 && k > 0 && (k % a.burst_every) == 0) n_arr += a.burst_size;
         }
+        const int n_w_old = n_w;
+        const uint32_t id0 = next_id;             // id of arrival 0 of this step
         for (int j = tid; j < n_arr; j += NT) {
-            const int pos = n_w + j;
+            const int pos = n_w_old + j;
             if (pos < W) {
                 const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)j >> 2, kStreamArrLen, 0u, key0, key1);
-                q_s[pos] = a.len_tab[word_of(r, j & 3) >> a.len_shift];
-                q_id[pos] = next_id + (uint32_t)j;
+                const int s = a.len_tab[word_of(r, j & 3) >> a.len_shift];
+                q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
             }
         }
-        const int n_w_old = n_w;
         int n_drop = n_w + n_arr - W;
         n_drop = n_drop > 0 ? n_drop : 0;
         n_w = n_w + n_arr - n_drop;
         next_id += (uint32_t)n_arr;
-        if (n_drop) status |= BR_ST_QUEUE_OVERFLOW;
-        __syncthreads();
+        if (timing) t_phase[1] = clock64();
 
-        // ================= PREDICT (H > 0) =================
+        // ============ PREDICT (H > 0): c_hat maintenance + horizon projection ============
         if (H > 0) {
             const bool warp_uniform = (B % 32) == 0;
-            const int A_up = (A + NT - 1) / NT * NT;
-            for (int s0 = tid; s0 < A_up; s0 += NT) {
-                const bool inr = s0 < A;
-                const int base = inr ? g_base[s0] : kEmpty;
-                const bool live = base != kEmpty;
-                int cur = 0, nh = -1;
-                if (live) {
-                    cur = base + k;
-                    const float c0 = g_chat0[s0];
-                    const int kr = g_kref[s0];
-                    const int t = (k - kr) & 255;
-                    float c = c0 - (float)t;
-                    if (t >= a.delta_T || c < a.c_floor) {
-                        const float *q = probs + (size_t)s0 * H;
-                        double surv = 1.0, cs = 0.0;
-                        for (int h = 0; h < H; ++h) {
-                            cs = __dadd_rn(cs, surv);
-                            surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
-                        }
-                        const double p_fin = __dsub_rn(1.0, surv);
-                        double v;
-                        if (p_fin >= (double)a.gate) {
-                            v = cs;
-                            if (v < (double)a.c_floor) v = (double)a.c_floor;
-                            if (v > (double)H) v = (double)H;
-                        } else {
-                            v = (double)H;
-                        }
-                        c = (float)v;
-                        g_chat0[s0] = c;
-                        g_kref[s0] = (uint8_t)(k & 255);
-                    }
-                    nh = (int)floorf(c);
-                    nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                }
-                const int g = (inr ? s0 : A - 1) / B;
-                if (warp_uniform) {
-                    for (int h = 0; h <= H; ++h) {
-                        const unsigned v = (live && h <= nh) ? (unsigned)(cur + h) : 0u;
-                        const unsigned s = __reduce_add_sync(kFull, v);
-                        if (lane == 0 && s)
-                            atomicAdd(reinterpret_cast<unsigned long long *>(&Lh[g * H1 + h]),
-                                      (unsigned long long)s);
-                    }
-                } else if (live) {
-                    for (int h = 0; h <= nh; ++h)
-                        atomicAdd(reinterpret_cast<unsigned long long *>(&Lh[g * H1 + h]),
-                                  (unsigned long long)(cur + h));
-                }
-            }
-            __syncthreads();
-        }
-        // envelope M_h = max_g L_g(k+h)
-        for (int h = tid; h < H1; h += NT) {
-            long long M = Lh[h];
-            for (int g = 1; g < G; ++g) M = max(M, Lh[g * H1 + h]);
-            Mh[h] = M;
-        }
-        // assign_out rows start at -1
-        for (int i = tid * 4; i < W; i += NT * 4)
-            *reinterpret_cast<int4 *>(assign + i) = make_int4(-1, -1, -1, -1);
-        __syncthreads();
-
-        Scorer<FP, HM> sc;
-
-        // optional F-score matrix before the first admission
-        if (a.out.fscore) {
-            double *F = a.out.fscore + orow * (size_t)W * G;
-            for (int g = 0; g < G; ++g) {
-                sc.load(Lh, Mh, g, H);
-                for (int i = tid; i < W; i += NT)
-                    F[(size_t)i * G + g] = (i < n_w) ? sc.value(sc.key(a, q_s[i])) : 0.0;
-            }
-        }
-
-        // ================= ROUTE =================
-        int S_tot = 0;
-        for (int g = 0; g < G; ++g) S_tot += cap[g];
-        int n_left = n_w;                      // waiting requests not yet admitted
-        const bool route = (S_tot > 0 && n_w > 0);
-
-        // commit request at queue position i (length s) to worker g; uniform across the block
-        auto commit = [&](int i, int s, int g) {
-            // every thread has finished reading the state it needs
-            __syncthreads();
-            if (tid == 0) {
-                int slot = -1;
-                for (int w = 0; w < OW && slot < 0; ++w) {
-                    const unsigned long long fr = ~occ[g * OW + w];
-                    if (fr) slot = w * 64 + __ffsll((long long)fr) - 1;
-                }
-                if (slot >= 0 && slot < B) {
-                    occ[g * OW + (slot >> 6)] |= 1ull << (slot & 63);
-                    cap[g] -= 1;
-                    for (int h = 0; h <= H; ++h) {
-                        const long long v = Lh[g * H1 + h] + s;
-                        Lh[g * H1 + h] = v;
-                        if (v > Mh[h]) Mh[h] = v;
-                    }
-                    const int sa = g * B + slot;
-                    g_base[sa] = s - k;
-                    if (g_aid) g_aid[sa] = q_id[i];
-                    if (H > 0) {
-                        g_chat0[sa] = (float)(H + a.delta_T - 1);
-                        g_kref[sa] = (uint8_t)((k + 1 - a.delta_T) & 255);
-                    }
-                    assign[i] = sa;
-                    scal[0] += 1;
-                } else {
-                    scal[3] |= BR_ST_BAD_STATE;
-                }
-                q_s[i] = -1;
-            }
-            __syncthreads();
-        };
-
-        // argmax_i F_g({i}) over all waiting requests, earliest position on ties
-        auto best_single = [&](int g) -> BestV {
-            sc.load(Lh, Mh, g, H);
-            long long bk = kNoKey; int bi = kNoIdx, bv = 0;
-            for (int i = tid; i < n_w; i += NT) {
-                const int s = q_s[i];
-                if (s < 0) continue;
-                const long long key = sc.key(a, s);
-                if (key > bk) { bk = key; bi = i; bv = s; }
-            }
-            return block_argmax_v(bk, bi, bv, red_key, red_idx, red_val, phase);
-        };
-
-        if (route) {
-            // ---------- Stage 1: greedy fill ----------
-            int guard_iters = 0;
-            while (S_tot > a.S_greedy && n_left > 0) {
-                if (++guard_iters > W) { status |= BR_ST_ITER_CAP; break; }
-                // worker with most free slots; ties: smallest L_g(k), then lowest g
-                Best bg{kNoKey, kNoIdx};
-                for (int g = lane; g < G; g += 32) {
-                    // key: cap (high), -(L) (low, loads < 2^31 by the create-time proof)
-                    const long long key = ((long long)cap[g] << 32) |
-                                          (long long)(0x7FFFFFFFu - (unsigned)Lh[g * H1]);
-                    if (key > bg.key) { bg.key = key; bg.idx = g; }
-                }
-                bg = warp_argmax(bg);
-                const int g = bg.idx;
-                const BestV bi = best_single(g);
-                if (bi.idx == kNoIdx) break;
-                commit(bi.idx, bi.val, g);
-                S_tot -= 1; n_left -= 1;
-                if (tid == 0) scal[1] += 1;
-            }
-
-            // ---------- Stage 2: refined allocation ----------
-            guard_iters = 0;
-            while (n_left > 0 && S_tot > 0) {
-                if (++guard_iters > W + G) { status |= BR_ST_ITER_CAP; break; }
-                // worker with (largest cap, largest horizon-min margin, lowest g), cap > 0
-                Best bg{kNoKey, kNoIdx};
-                for (int g = lane; g < G; g += 32) {
-                    if (cap[g] <= 0) continue;
-                    long long mm = Mh[0] - Lh[g * H1];
-                    for (int h = 1; h <= H; ++h) mm = min(mm, Mh[h] - Lh[g * H1 + h]);
-                    const long long key = ((long long)cap[g] << 32) | (long long)(unsigned)mm;
-                    if (key > bg.key) { bg.key = key; bg.idx = g; }
-                }
-                bg = warp_argmax(bg);
-                if (bg.idx == kNoIdx) break;
-                const int g = bg.idx;
-                if (tid == 0) scal[2] += 1;
-
-                // window: the R_max largest waiting requests, earliest first on ties
-                int win_i[BR_MAX_RMAX], win_s[BR_MAX_RMAX];
-                int nwin = 0;
-                long long prev = 0x7FFFFFFFFFFFFFFFll;
+            for (int s_base = 0; s_base < A; s_base += NT * kUnroll) {
+                int bs[kUnroll]; float c0s[kUnroll]; int krs[kUnroll];
 #pragma unroll
-                for (int r = 0; r < BR_MAX_RMAX; ++r) {
-                    if (r < a.R_max && r < n_left) {
-                        long long bk = kNoKey; int bi = kNoIdx, bv = 0;
-                        for (int i = tid; i < n_w; i += NT) {
-                            const int s = q_s[i];
-                            if (s < 0) continue;
-                            const long long key = ((long long)s << 32) | (long long)(unsigned)(0x7FFFFFFF - i);
-                            if (key < prev && key > bk) { bk = key; bi = i; bv = s; }
+                for (int u = 0; u < kUnroll; ++u) {
+                    const int s0 = s_base + u * NT + tid;
+                    const bool inr = s0 < A;
+                    bs[u] = inr ? g_base[s0] : kEmpty;
+                    c0s[u] = inr ? g_chat0[s0] : 0.0f;
+                    krs[u] = inr ? (int)g_kref[s0] : 0;
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const int s0 = s_base + u * NT + tid;
+                    if (s_base + u * NT >= A) break;               // uniform across the block
+                    const bool inr = s0 < A;
+                    const bool live = bs[u] != kEmpty;
+                    int cur = 0, nh = -1;
+                    if (live) {
+                        cur = bs[u] + k;
+                        const int t = (k - krs[u]) & 255;
+                        float c = c0s[u] - (float)t;
+                        if (t >= a.delta_T || c < a.c_floor) {
+                            const float *q = probs + (size_t)s0 * H;
+                            double surv = 1.0, cs = 0.0;
+                            if ((H & 3) == 0) {
+                                for (int h = 0; h < H; h += 4) {
+                                    const float4 qq = *reinterpret_cast<const float4 *>(q + h);
+                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.x));
+                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.y));
+                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.z));
+                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.w));
+                                }
+                            } else {
+                                for (int h = 0; h < H; ++h) {
+                                    cs = __dadd_rn(cs, surv);
+                                    surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
+                                }
+                            }
+                            const double p_fin = __dsub_rn(1.0, surv);
+                            double v;
+                            if (p_fin >= (double)a.gate) {
+                                v = cs;
+                                if (v < (double)a.c_floor) v = (double)a.c_floor;
+                                if (v > (double)H) v = (double)H;
+                            } else {
+                                v = (double)H;
+                            }
+                            c = (float)v;
+                            g_chat0[s0] = c;
+                            g_kref[s0] = (uint8_t)(k & 255);
                         }
-                        const BestV w = block_argmax_v(bk, bi, bv, red_key, red_idx, red_val, phase);
-                        win_i[r] = w.idx; win_s[r] = w.val; prev = w.key;
-                        if (w.idx != kNoIdx) nwin = r + 1;
+                        nh = (int)floorf(c);
+                        nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                    }
+                    const int g = (inr ? s0 : A - 1) / B;
+                    if (warp_uniform) {
+                        for (int h = 0; h <= H; ++h) {
+                            const unsigned v = (live && h <= nh) ? (unsigned)(cur + h) : 0u;
+                            const unsigned s = __reduce_add_sync(kFull, v);
+                            if (lane == 0 && s) atomicAdd(&Lh_s[g * H1 + h], s);
+                        }
+                    } else if (live) {
+                        for (int h = 0; h <= nh; ++h) atomicAdd(&Lh_s[g * H1 + h], (unsigned)(cur + h));
+                    }
+                }
+            }
+        }
+        __syncthreads();                                              // B1
+        if (timing) t_phase[2] = clock64();
+
+        if (warp == 0) {
+            // ================= ROUTE (warp 0 only, warp-synchronous) =================
+            if (H > 0) {
+#pragma unroll
+                for (int w = 0; w < GW; ++w) {
+                    const int g = lane + 32 * w;
+#pragma unroll
+                    for (int h = 0; h <= HM; ++h)
+                        L[w][h] = (g < G && h <= H) ? (int)Lh_s[g * H1 + h] : 0;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h <= HM; ++h) {
+                int v = L[0][h];
+#pragma unroll
+                for (int w = 1; w < GW; ++w) v = max(v, L[w][h]);
+                Mh[h] = (h <= H) ? __reduce_max_sync(kFull, v) : 0;
+            }
+
+            Scorer<FP, HM> sc;
+            // margins of worker g -> every lane's scorer
+            auto load_margins = [&](int g) {
+                const int src = g & 31;
+                const int set = g >> 5;
+                if (!FP) {
+                    int mine = Mh[0] - L[0][0];
+#pragma unroll
+                    for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[0] - L[w][0];
+                    sc.mi = __shfl_sync(kFull, mine, src);
+                } else {
+#pragma unroll
+                    for (int h = 0; h <= HM; ++h) {
+                        int mine = Mh[h] - L[0][h];
+#pragma unroll
+                        for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[h] - L[w][h];
+                        sc.md[h] = (double)__shfl_sync(kFull, mine, src);
+                    }
+                }
+            };
+
+            // optional F-score matrix before the first admission
+            if (a.out.fscore) {
+                double *F = a.out.fscore + orow * (size_t)W * G;
+                for (int g = 0; g < G; ++g) {
+                    load_margins(g);
+                    for (int i = lane; i < W; i += 32)
+                        F[(size_t)i * G + g] = (i < n_w) ? sc.value(sc.key(a, q_key[i] >> WL)) : 0.0;
+                }
+            }
+
+            int S_tot = 0;
+#pragma unroll
+            for (int w = 0; w < GW; ++w) S_tot += cap[w] > 0 ? cap[w] : 0;
+            S_tot = (int)__reduce_add_sync(kFull, (unsigned)S_tot);
+            int n_left = n_w;
+            int admitted = 0, s1_iters = 0, s2_pops = 0, status = 0;
+            const int n_tiles = (n_w + 31) >> 5;
+
+            // argmax_i F_g({i}) over all waiting requests, earliest arrival on ties.
+            // Returns the packed key of the winner (0 if none).
+            auto best_single = [&]() -> int {
+                long long bk = kNoKey; unsigned bt = 0; int bkey = 0;
+                for (int t = 0; t < n_tiles; ++t) {
+                    const int idx = (t << 5) + lane;
+                    const int qk = idx < n_w ? q_key[idx] : 0;
+                    if (qk > 0) {
+                        const long long f = sc.key(a, qk >> WL);
+                        const unsigned tie = (unsigned)qk & posmask;      // larger = earlier
+                        if (f > bk || (f == bk && tie > bt)) { bk = f; bt = tie; bkey = qk; }
+                    }
+                }
+                long long wk;
+                const int src = warp_argmax_lane(bk, bt, wk);
+                const int res = __shfl_sync(kFull, bkey, src);
+                return wk == kNoKey ? 0 : res;
+            };
+
+            // sticky admission of the request with packed key qk to worker g
+            auto commit = [&](int qk, int g) {
+                const int s = qk >> WL;
+                const int pos = (int)(posmask - ((unsigned)qk & posmask));
+                const int src = g & 31, set = g >> 5;
+                if (lane == src) {
+                    int slot = -1;
+                    for (int w = 0; w < OW && slot < 0; ++w) {
+                        const unsigned long long fr = ~occ[g * OW + w];
+                        if (fr) slot = w * 64 + __ffsll((long long)fr) - 1;
+                    }
+                    if (slot >= 0 && slot < B) {
+                        occ[g * OW + (slot >> 6)] |= 1ull << (slot & 63);
+                        const int sa = g * B + slot;
+                        g_base[sa] = s - k;
+                        if (H > 0) {
+                            g_chat0[sa] = (float)(H + a.delta_T - 1);
+                            g_kref[sa] = (uint8_t)((k + 1 - a.delta_T) & 255);
+                        }
+                        q_key[pos] = (int)(0x80000000u | (unsigned)sa);
                     } else {
-                        win_i[r] = kNoIdx; win_s[r] = 0;
+                        status |= BR_ST_BAD_STATE;
+                        q_key[pos] = -1;                  // gone, no slot
+                    }
+#pragma unroll
+                    for (int w = 0; w < GW; ++w) {
+                        if (set == w) {
+                            cap[w] -= 1;
+#pragma unroll
+                            for (int h = 0; h <= HM; ++h) if (h <= H) L[w][h] += s;
+                        }
                     }
                 }
-                // subsets: lane = mask
-                const int lim = min(cap[g], a.R_max);
-                sc.load(Lh, Mh, g, H);
-                Best bm{kNoKey, kNoIdx};
-                if (lane >= 1 && lane < (1 << nwin) && __popc(lane) <= lim) {
-                    int delta = 0;
+                // envelope: only worker g grew, so M_h = max(M_h, L_g(k+h))
 #pragma unroll
-                    for (int r = 0; r < BR_MAX_RMAX; ++r)
-                        if ((lane >> r) & 1) delta += win_s[r];
-                    bm.key = sc.key(a, delta);
-                    bm.idx = lane;
+                for (int h = 0; h <= HM; ++h) {
+                    if (h <= H) {
+                        int mine = L[0][h];
+#pragma unroll
+                        for (int w = 1; w < GW; ++w) if (set == w) mine = L[w][h];
+                        Mh[h] = max(Mh[h], __shfl_sync(kFull, mine, src));
+                    }
                 }
-                bm = warp_argmax(bm);
-                if (bm.idx == kNoIdx) { status |= BR_ST_ITER_CAP; break; }
-                if (bm.key <= 0) {
-                    // starvation guard: least-bad single request of all of R_wait
-                    const BestV bi = best_single(g);
-                    if (bi.idx == kNoIdx) break;
-                    commit(bi.idx, bi.val, g);
-                    S_tot -= 1; n_left -= 1;
-                } else {
+                __syncwarp();
+                S_tot -= 1; n_left -= 1; admitted += 1;
+            };
+
+            if (S_tot > 0 && n_w > 0) {
+                // ---------- Stage 1: greedy fill ----------
+                while (S_tot > a.S_greedy && n_left > 0) {
+                    if (s1_iters >= W) { status |= BR_ST_ITER_CAP; break; }
+                    ++s1_iters;
+                    // most free slots; ties: smallest L_g(k), then lowest g
+                    int bc = cap[0], bl = L[0][0], bg = lane;
+#pragma unroll
+                    for (int w = 1; w < GW; ++w)
+                        if (cap[w] > bc || (cap[w] == bc && L[w][0] < bl)) { bc = cap[w]; bl = L[w][0]; bg = lane + 32 * w; }
+                    const int mc = __reduce_max_sync(kFull, bc);
+                    const unsigned ml = __reduce_min_sync(kFull, bc == mc ? (unsigned)bl : 0xFFFFFFFFu);
+                    const unsigned mg = __reduce_min_sync(kFull, (bc == mc && (unsigned)bl == ml) ? (unsigned)bg : 0xFFFFFFFFu);
+                    const int g = (int)mg;
+                    load_margins(g);
+                    const int qk = best_single();
+                    if (qk <= 0) break;
+                    commit(qk, g);
+                }
+            }
+            if (timing) t_phase[3] = clock64();
+            if (S_tot > 0 && n_left > 0) {
+                // ---------- Stage 2: refined allocation ----------
+                while (n_left > 0 && S_tot > 0) {
+                    if (s2_pops >= W + G) { status |= BR_ST_ITER_CAP; break; }
+                    ++s2_pops;
+                    // (largest cap, largest horizon-min margin, lowest g) among cap > 0
+                    int bc = -1, bm = -1, bg = 0x7FFFFFFF;
+#pragma unroll
+                    for (int w = 0; w < GW; ++w) {
+                        int mm = Mh[0] - L[w][0];
+#pragma unroll
+                        for (int h = 1; h <= HM; ++h) if (h <= H) mm = min(mm, Mh[h] - L[w][h]);
+                        if (cap[w] > 0 && (cap[w] > bc || (cap[w] == bc && mm > bm))) { bc = cap[w]; bm = mm; bg = lane + 32 * w; }
+                    }
+                    const int mc = __reduce_max_sync(kFull, bc);
+                    if (mc <= 0) break;
+                    const int mm2 = __reduce_max_sync(kFull, bc == mc ? bm : -1);
+                    const unsigned mg = __reduce_min_sync(kFull, (bc == mc && bm == mm2) ? (unsigned)bg : 0xFFFFFFFFu);
+                    const int g = (int)mg;
+                    load_margins(g);
+
+                    // window: the R_max largest waiting requests, earliest first on ties
+                    int win[BR_MAX_RMAX];
+                    int nwin = 0;
+                    int prev = 0x7FFFFFFF;
 #pragma unroll
                     for (int r = 0; r < BR_MAX_RMAX; ++r) {
-                        if ((bm.idx >> r) & 1) {
-                            commit(win_i[r], win_s[r], g);
-                            S_tot -= 1; n_left -= 1;
+                        win[r] = 0;
+                        if (r < a.R_max && r < n_left) {
+                            int best = 0;
+                            for (int t = 0; t < n_tiles; ++t) {
+                                const int idx = (t << 5) + lane;
+                                const int qk = idx < n_w ? q_key[idx] : 0;
+                                if (qk < prev && qk > best) best = qk;
+                            }
+                            best = __reduce_max_sync(kFull, best);
+                            win[r] = best; prev = best;
+                            if (best > 0) nwin = r + 1;
                         }
                     }
+                    // subsets of the window: lane = mask, lowest mask on ties
+                    const int lim = min(mc, a.R_max);
+                    long long fk = kNoKey;
+                    if (lane >= 1 && lane < (1 << nwin) && __popc(lane) <= lim) {
+                        int delta = 0;
+#pragma unroll
+                        for (int r = 0; r < BR_MAX_RMAX; ++r)
+                            if ((lane >> r) & 1) delta += win[r] >> WL;
+                        fk = sc.key(a, delta);
+                    }
+                    long long wk;
+                    const int best_mask = warp_argmax_lane(fk, 31u - (unsigned)lane, wk);
+                    if (wk == kNoKey) { status |= BR_ST_ITER_CAP; break; }
+                    if (wk <= 0) {
+                        // starvation guard: least-bad single request of all of R_wait
+                        const int qk = best_single();
+                        if (qk <= 0) break;
+                        commit(qk, g);
+                    } else {
+#pragma unroll
+                        for (int r = 0; r < BR_MAX_RMAX; ++r)
+                            if ((best_mask >> r) & 1) commit(win[r], g);
+                    }
                 }
             }
-        }
-        __syncthreads();
+            if (timing) t_phase[4] = clock64();
 
-        // ================= RECORD =================
-        {
-            Best mx{kNoKey, kNoIdx}, mn{kNoKey, kNoIdx};
-            long long sum = 0;
-            for (int g = lane; g < G; g += 32) {
-                const long long L = Lh[g * H1];
-                if (L > mx.key || mx.idx == kNoIdx) { mx.key = L; mx.idx = g; }
-                if (-L > mn.key || mn.idx == kNoIdx) { mn.key = -L; mn.idx = g; }
-                sum += L;
+            // ================= RECORD =================
+            {
+                int mx = L[0][0], mn = cap[0] >= 0 ? L[0][0] : 0x7FFFFFFF;
+                long long sum = cap[0] >= 0 ? (long long)L[0][0] : 0;
+                long long *o_load = reinterpret_cast<long long *>(a.out.load) + orow * G;
+                if (cap[0] >= 0) o_load[lane] = L[0][0];
+#pragma unroll
+                for (int w = 1; w < GW; ++w) {
+                    if (cap[w] >= 0) {
+                        mx = max(mx, L[w][0]); mn = min(mn, L[w][0]); sum += L[w][0];
+                        o_load[lane + 32 * w] = L[w][0];
+                    }
+                }
+                mx = __reduce_max_sync(kFull, mx);
+                mn = __reduce_min_sync(kFull, mn);
+                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+                status = (int)__reduce_or_sync(kFull, (unsigned)status);
+                if (lane == 0) {
+                    long long *tr = reinterpret_cast<long long *>(a.out.trace) + orow * 3;
+                    tr[0] = mx; tr[1] = mn; tr[2] = sum;
+                    scal[0] = n_left; scal[1] = admitted; scal[2] = s1_iters; scal[3] = s2_pops;
+                    scal[4] = status | (n_drop ? BR_ST_QUEUE_OVERFLOW : 0);
+                }
             }
-            mx = warp_argmax(mx);
-            mn = warp_argmax(mn);
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
-            long long *o_load = reinterpret_cast<long long *>(a.out.load) + orow * G;
-            for (int g = tid; g < G; g += NT) o_load[g] = Lh[g * H1];
-            if (tid == 0) {
-                long long *tr = reinterpret_cast<long long *>(a.out.trace) + orow * 3;
-                tr[0] = mx.key; tr[1] = -mn.key; tr[2] = sum;
+        } else if (a.term_mode == 1) {
+            // warps 1.. draw this step's termination words while warp 0 routes
+            const int A4 = A >> 2;
+            for (int q4 = tid - 32; q4 < A4; q4 += NT - 32) {
+                const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
+                term_nib[q4] = (unsigned char)((r.x < a.hazard_thr ? 1 : 0) | (r.y < a.hazard_thr ? 2 : 0) |
+                                               (r.z < a.hazard_thr ? 4 : 0) | (r.w < a.hazard_thr ? 8 : 0));
             }
         }
+        __syncthreads();                                              // B2: admissions visible
 
-        // ================= queue compaction (stable, in shared memory) =================
-        if (tid < 32 && n_left != n_w) {
+        // ============ queue compaction, assignments, ids of admitted requests (warp 0) ============
+        if (warp == 0) {
+            int32_t *assign = a.assign_out + orow * W;
             int run = 0;
-            for (int i0 = 0; i0 < n_w; i0 += 32) {
+            const int n_before = n_w;          // queue length after ARRIVE
+            for (int i0 = 0; i0 < W; i0 += 32) {
                 const int i = i0 + lane;
-                const int s = (i < n_w) ? q_s[i] : -1;
-                const unsigned id = (i < n_w) ? q_id[i] : 0u;
-                const bool keep = s >= 0;
+                const bool inq = i < n_before;
+                const int qk = inq ? q_key[i] : 0;
+                const bool gone = inq && qk < 0;
+                const bool keep = inq && qk > 0;
                 const unsigned bal = __ballot_sync(kFull, keep);
                 const int dst = run + __popc(bal & ((1u << lane) - 1u));
+                const int sa = qk & 0x7FFFFFFF;
+                if (i < W) assign[i] = (gone && sa < A) ? sa : -1;
+                unsigned id = 0;
+                const bool fresh = i >= n_w_old;                  // arrived this step
+                const bool moved = keep && (dst != i || fresh);
+                if (!fresh && ((gone && g_aid) || moved)) id = g_qid[i];
+                if (fresh) id = id0 + (unsigned)(i - n_w_old);
                 __syncwarp();
-                if (keep && dst != i) { q_s[dst] = s; q_id[dst] = id; }
+                if (gone && g_aid && sa < A) g_aid[sa] = id;
+                if (keep) {
+                    const int s = qk >> WL;
+                    q_key[dst] = (s << WL) | (int)(posmask - (unsigned)dst);
+                    if (moved) { g_qs[dst] = s; g_qid[dst] = id; }
+                }
                 __syncwarp();
                 run += __popc(bal);
+                if (i0 + 32 >= n_before) {
+                    // the rest of the row is beyond the queue: only assignments remain
+                    for (int j = i0 + 32 + lane; j < W; j += 32) assign[j] = -1;
+                    break;
+                }
             }
         }
-        n_w = n_left;
-        __syncthreads();
+        n_w = scal[0];
+        if (timing) t_phase[5] = clock64();
 
-        // ================= ADVANCE =================
-        for (int g = tid; g < G; g += NT) { load_new[g] = 0; nact_new[g] = 0; }
-        __syncthreads();
+        // ================= ADVANCE (all warps) =================
         {
             const int A4 = A >> 2;
-            const int A4_up = (A4 + NT - 1) / NT * NT;
-            for (int q4 = tid; q4 < A4_up; q4 += NT) {
-                const bool inr = q4 < A4;
-                int4 b = make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
-                if (inr) b = *reinterpret_cast<const int4 *>(g_base + q4 * 4);
-                const bool any = (b.x != kEmpty) | (b.y != kEmpty) | (b.z != kEmpty) | (b.w != kEmpty);
-                unsigned part = 0; int cnt = 0; unsigned ended = 0;
-                if (any) {
-                    uint4 r = make_uint4(0, 0, 0, 0);
-                    if (a.term_mode != 0)
-                        r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
-                    int bb[4] = {b.x, b.y, b.z, b.w};
-                    const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
+            const bool pre = (nwarps > 1) && a.term_mode == 1;
+            for (int q_base = 0; q_base < A4; q_base += NT * kUnroll) {
+                int4 bv[kUnroll];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (bb[j] == kEmpty) continue;
-                        bool fin = false;
-                        if (a.term_mode == 1) fin = rr[j] < a.hazard_thr;
-                        else if (a.term_mode == 2)
-                            fin = __fmul_rn((float)(rr[j] >> 8), 5.9604644775390625e-8f) <
-                                  probs[(size_t)(q4 * 4 + j) * H];
-                        if (fin) { ended |= 1u << j; bb[j] = kEmpty; }
-                        else { part += (unsigned)(bb[j] + k + 1); cnt += 1; }
+                for (int u = 0; u < kUnroll; ++u) {
+                    const int q4 = q_base + u * NT + tid;
+                    bv[u] = make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
+                    if (q4 < A4) bv[u] = *reinterpret_cast<const int4 *>(g_base + q4 * 4);
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (q_base + u * NT >= A4) break;              // uniform across the block
+                    const int q4 = q_base + u * NT + tid;
+                    const bool inr = q4 < A4;
+                    const int4 b = bv[u];
+                    const bool any = (b.x != kEmpty) | (b.y != kEmpty) | (b.z != kEmpty) | (b.w != kEmpty);
+                    unsigned part = 0, ended = 0; int cnt = 0;
+                    if (any) {
+                        unsigned fin = 0;
+                        if (a.term_mode == 1) {
+                            if (pre) {
+                                fin = term_nib[q4];
+                            } else {
+                                const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
+                                fin = (r.x < a.hazard_thr ? 1u : 0u) | (r.y < a.hazard_thr ? 2u : 0u) |
+                                      (r.z < a.hazard_thr ? 4u : 0u) | (r.w < a.hazard_thr ? 8u : 0u);
+                            }
+                        } else if (a.term_mode == 2) {
+                            const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
+                            const float *q = probs + (size_t)q4 * 4 * H;
+                            const float sc24 = 5.9604644775390625e-8f;
+                            fin = (__fmul_rn((float)(r.x >> 8), sc24) < q[0] ? 1u : 0u) |
+                                  (__fmul_rn((float)(r.y >> 8), sc24) < q[H] ? 2u : 0u) |
+                                  (__fmul_rn((float)(r.z >> 8), sc24) < q[2 * H] ? 4u : 0u) |
+                                  (__fmul_rn((float)(r.w >> 8), sc24) < q[3 * H] ? 8u : 0u);
+                        }
+                        int bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (bb[j] == kEmpty) continue;
+                            if ((fin >> j) & 1u) { ended |= 1u << j; bb[j] = kEmpty; }
+                            else { part += (unsigned)(bb[j] + k + 1); cnt += 1; }
+                        }
+                        if (ended) *reinterpret_cast<int4 *>(g_base + q4 * 4) = make_int4(bb[0], bb[1], bb[2], bb[3]);
                     }
-                    if (ended) *reinterpret_cast<int4 *>(g_base + q4 * 4) = make_int4(bb[0], bb[1], bb[2], bb[3]);
-                }
-                const int g = (inr ? q4 * 4 : A - 4) / B;
-                // segmented sums over lanes of the same worker
-                const unsigned peers = __match_any_sync(kFull, g);
-                const unsigned psum = __reduce_add_sync(peers, part);
-                const int pcnt = (int)__reduce_add_sync(peers, (unsigned)cnt);
-                if (lane == __ffs(peers) - 1 && inr) {
-                    if (psum) atomicAdd(reinterpret_cast<unsigned long long *>(&load_new[g]), (unsigned long long)psum);
-                    if (pcnt) atomicAdd(&nact_new[g], pcnt);
-                }
-                if (ended) {
-                    const int slot0 = (q4 * 4) % B;
-                    atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
+                    const int g = (inr ? q4 * 4 : A - 4) / B;
+                    // segmented sums over the lanes that hold the same worker
+                    unsigned peers;
+                    if ((B & 127) == 0) peers = kFull;
+                    else if (B == 64) peers = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
+                    else peers = __match_any_sync(kFull, g);
+                    const unsigned psum = __reduce_add_sync(peers, part);
+                    const int pcnt = (int)__reduce_add_sync(peers, (unsigned)cnt);
+                    if (lane == __ffs(peers) - 1 && inr && pcnt) {
+                        atomicAdd(&load_new[g], psum);
+                        atomicAdd(&nact_new[g], pcnt);
+                    }
+                    if (ended) {
+                        const int slot0 = (q4 * 4) % B;
+                        atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
+                    }
                 }
             }
         }
-        __syncthreads();
-        for (int g = tid; g < G; g += NT) {
-            cap[g] = B - nact_new[g];
-            if (H == 0) Lh[g] = load_new[g];
-        }
-        if (tid == 0) {
-            if (a.out.counters) {
-                uint32_t *c = a.out.counters + orow * 4;
-                c[0] = (uint32_t)n_drop; c[1] = (uint32_t)scal[0]; c[2] = (uint32_t)scal[1]; c[3] = (uint32_t)scal[2];
+        __syncthreads();                                              // B3
+
+        if (warp == 0) {
+#pragma unroll
+            for (int w = 0; w < GW; ++w) {
+                const int g = lane + 32 * w;
+                if (g < G) {
+                    cap[w] = B - nact_new[g];
+                    L[w][0] = (int)load_new[g];
+                }
             }
-            if (a.out.status) a.out.status[orow] = status | scal[3] | scal[4];
+            if (lane == 0) {
+                if (a.out.counters) {
+                    uint32_t *c = a.out.counters + orow * 4;
+                    c[0] = (uint32_t)n_drop; c[1] = (uint32_t)scal[1]; c[2] = (uint32_t)scal[2]; c[3] = (uint32_t)scal[3];
+                }
+                if (a.out.status) a.out.status[orow] = scal[4] | scal[5];
+                if (timing) {
+                    t_phase[6] = clock64();
+                    uint32_t *pc = a.out.phase_cycles + orow * 6;
+#pragma unroll
+                    for (int p = 0; p < 6; ++p) pc[p] = (uint32_t)(t_phase[p + 1] - t_phase[p]);
+                }
+            }
+            __syncwarp();
+            if (it + 1 < a.n_steps) {
+                for (int i = lane; i < G; i += 32) { load_new[i] = 0u; nact_new[i] = 0; }
+            }
         }
-        status = 0;
-        __syncthreads();
+        if (it + 1 < a.n_steps) {
+            for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
+            __syncthreads();
+        }
     }
 
     // ---- write the snapshot back ----
-    for (int g = tid; g < G; g += NT) {
-        g_load[g] = load_new[g];
-        g_nact[g] = nact_new[g];
+    if (warp == 0) {
+#pragma unroll
+        for (int w = 0; w < GW; ++w) {
+            const int g = lane + 32 * w;
+            if (g < G) { g_load[g] = (long long)L[w][0]; g_nact[g] = B - cap[w]; }
+        }
     }
     for (int i = tid; i < G * OW; i += NT) g_occ[i] = occ[i];
-    for (int i = tid * 4; i < n_w; i += NT * 4) {
-        *reinterpret_cast<int4 *>(g_qs + i) = *reinterpret_cast<const int4 *>(q_s + i);
-        *reinterpret_cast<uint4 *>(g_qid + i) = *reinterpret_cast<const uint4 *>(q_id + i);
-    }
     if (tid == 0) {
         a.ws.step[inst] = k;
         a.ws.next_id[inst] = next_id;
