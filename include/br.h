@@ -41,7 +41,7 @@ extern "C" {
 /* compiled limits */
 #define BR_MAX_G      64
 #define BR_MAX_H      16
-#define BR_MAX_B     256     /* B must be a multiple of 4                     */
+#define BR_MAX_B     256     /* B must be a multiple of 8                     */
 #define BR_MAX_W    4096     /* W must be a multiple of 4                     */
 #define BR_MAX_RMAX    5     /* Stage 2 enumerates 2^R_max - 1 <= 31 subsets   */
 
@@ -68,8 +68,9 @@ typedef struct {
     float   gate;           /* confidence gate on p_fin; < 0 -> 0.5                          */
     float   c_floor;        /* lower bound of c_hat; < 0 -> 1                                */
     int32_t score_mode;     /* 0: Eq. 1 in integers (needs H == 0); 1: Eq. 2 in fp64; < 0 -> 0 if H == 0 else 1 */
-    int32_t term_mode;      /* 0: requests never end; 1: end when Philox word < hazard_thr;
-                               2: end when 24-bit Philox uniform < term_probs[slot][0]       */
+    int32_t term_mode;      /* 0: requests never end; 1: end with probability hazard_thr / 2^32 per step
+                               (16 Philox bits per slot, 16 more when they tie with the threshold);
+                               2: end when a 24-bit Philox uniform < term_probs[slot][0]     */
     uint32_t hazard_thr;
     const uint32_t *arr_cdf;/* device [rows][arr_len] Poisson CDF thresholds; the row for instance i
                                at step k is i * arr_inst_stride + k % arr_period; NULL -> no arrivals */

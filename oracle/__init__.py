@@ -59,6 +59,8 @@ def lib():
         L.orc_projection.argtypes = [C.c_void_p] + [C.c_void_p] * 3
         L.orc_predict_only.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_philox4x32_10.argtypes = [C.c_void_p] * 3
+        L.orc_term_decision.restype = C.c_int
+        L.orc_term_decision.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32]
         L.orc_f_br0.restype = C.c_int64
         L.orc_f_br0.argtypes = [C.c_int32, C.c_int64, C.c_int64]
         L.orc_f_brh.restype = C.c_double
@@ -90,6 +92,10 @@ def philox4x32_10(ctr, key) -> np.ndarray:
     out = np.zeros(4, dtype=np.uint32)
     lib().orc_philox4x32_10(_p(c), _p(k), _p(out))
     return out
+
+
+def term_decision(v16: int, w16: int, thr: int) -> bool:
+    return bool(lib().orc_term_decision(v16, w16, thr))
 
 
 def f_br0(G: int, delta: int, m: int) -> int:

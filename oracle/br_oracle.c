@@ -98,7 +98,7 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2 };
+enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2, STREAM_TERM_REFINE = 3 };
 
 static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
 {
@@ -108,6 +108,37 @@ static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
     return out[entity & 3u];
+}
+
+/*
+ * Constant-hazard termination of the request in slot a at step k: a Bernoulli event of
+ * probability thr / 2^32 realised from 16 + 16 Philox bits.  The first 16 bits v are
+ * half j % 2 of word j / 2 (j = a % 8) of the block with counter (k, a / 8, TERM, 0);
+ * they decide unless v equals the high half of thr, in which case the low 16 bits of
+ * word 0 of the block (k, a, TERM_REFINE, 0) are compared with the low half of thr.
+ * READING: the paper fixes only the per-step probability (Section 2.2 leaves o_i latent);
+ * the bit recipe is this workload's, chosen so that one Philox block serves 8 slots.
+ */
+int orc_term_decision(uint32_t v16, uint32_t w16, uint32_t thr)
+{
+    uint32_t hi = thr >> 16, lo = thr & 0xFFFFu;
+    return v16 < hi || (v16 == hi && w16 < lo);
+}
+
+static int hazard_fin(const orc_inst *s, uint32_t a)
+{
+    uint32_t key[2] = { (uint32_t)s->seed, (uint32_t)(s->seed >> 32) };
+    uint32_t ctr[4] = { (uint32_t)s->k, a >> 3, STREAM_TERM, 0u };
+    uint32_t out[4], ref[4];
+    orc_philox4x32_10(ctr, key, out);
+    uint32_t j = a & 7u;
+    uint32_t v16 = (out[j >> 1] >> (16u * (j & 1u))) & 0xFFFFu;
+    ref[0] = 0u;
+    if (v16 == (s->p.hazard_thr >> 16)) {          /* the second draw matters only on equality */
+        uint32_t ctr2[4] = { (uint32_t)s->k, a, STREAM_TERM_REFINE, 0u };
+        orc_philox4x32_10(ctr2, key, ref);
+    }
+    return orc_term_decision(v16, ref[0] & 0xFFFFu, s->p.hazard_thr);
 }
 
 /* ------------------------------------------------------------------ */
@@ -557,7 +588,7 @@ void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
         if (!s->occ[a]) continue;
         int fin = 0;
         if (p->term_mode == 1) {
-            fin = draw(s, (uint32_t)a, STREAM_TERM) < p->hazard_thr;
+            fin = hazard_fin(s, (uint32_t)a);
         } else if (p->term_mode == 2) {
             uint32_t u = draw(s, (uint32_t)a, STREAM_TERM) >> 8;       /* 24 bits */
             fin = ((float)u * 5.9604644775390625e-8f) < probs[(size_t)a * p->H];

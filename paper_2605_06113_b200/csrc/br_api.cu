@@ -130,7 +130,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     if (!params || !out) return BR_EINVAL;
     if (G < 1 || G > BR_MAX_G || H < 0 || H > BR_MAX_H) return BR_EINVAL;
     br_params p = *params;
-    if (p.B < 4 || p.B > BR_MAX_B || (p.B % 4) != 0) return BR_EINVAL;
+    if (p.B < 8 || p.B > BR_MAX_B || (p.B % 8) != 0) return BR_EINVAL;
     if (p.W < 4 || p.W > BR_MAX_W || (p.W % 4) != 0) return BR_EINVAL;
     if (p.R_max <= 0) p.R_max = 4;
     if (p.R_max > BR_MAX_RMAX) return BR_EINVAL;

@@ -8,9 +8,12 @@
 // sequential admission loop with warp reductions only: no block barrier sits on the
 // admission chain.  The waiting queue lives in shared memory as packed 32-bit keys
 // (prompt length in the high bits, inverted position in the low bits) so that "largest
-// s, earliest arrival" is one integer max.  All warps stream the running-request state
-// (PREDICT, ADVANCE) with coalesced 16-byte loads issued in batches; while warp 0 routes,
-// the other warps already draw the Philox termination words of the step.
+// s, earliest arrival" is one integer max.
+//
+// Loads are advanced incrementally: L_g(k+1) = L_g(k) - sum of the loads of the requests
+// that end at k + number of survivors, so ADVANCE touches only the occupancy bit masks,
+// one Philox block per 8 slots, and the few slots whose request ends.  Only the horizon
+// projection of BR-H streams the per-request state.
 #pragma once
 #include "br_device.cuh"
 #include "../../include/br.h"
@@ -43,11 +46,11 @@ struct StepArgs {
 __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words)
 {
     size_t n = 0;
-    n += 4 * (size_t)W;                          // q_key
+    n += 4 * (size_t)W * 2;                      // q_key, q_id
     n += 8 * (size_t)G * occ_words;              // occ
     n += 4 * (size_t)G * (H + 1);                // Lh_s (PREDICT accumulators)
-    n += 4 * (size_t)G * 2;                      // load_new, nact_new
-    n += ((size_t)G * B / 4 + 15) & ~(size_t)15; // term_nib
+    n += 4 * (size_t)G;                          // sub_load
+    n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
     n += 64;                                     // scalars
     return (n + 15) & ~(size_t)15;
 }
@@ -100,7 +103,24 @@ __device__ __forceinline__ int warp_argmax_lane(long long key, unsigned tie, lon
     return __ffs(who) - 1;
 }
 
-constexpr int kUnroll = 4;      // 16-byte loads in flight per thread in the streaming phases
+// same for 32-bit keys (Eq. 1 scores): largest key, then largest tie value
+__device__ __forceinline__ int warp_argmax_lane32(int key, unsigned tie, int &wkey)
+{
+    const int mk = __reduce_max_sync(kFull, key);
+    const bool in1 = key == mk;
+    const unsigned mt = __reduce_max_sync(kFull, in1 ? tie : 0u);
+    const unsigned who = __ballot_sync(kFull, in1 && tie == mt);
+    wkey = mk;
+    return __ffs(who) - 1;
+}
+
+// nonzero iff some 16-bit field of x is below n (n <= 0x8000)
+__device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
+{
+    return (x - 0x00010001u * n) & ~x & 0x80008000u;
+}
+
+constexpr int kUnroll = 4;      // loads in flight per thread in the BR-H streaming phase
 
 template <bool FP, int HM, int GW>
 __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
@@ -109,18 +129,21 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
     const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5;
     const int nwarps = NT >> 5;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
+    const int A8 = A >> 3;
     const int WL = a.wl;
     const unsigned posmask = (1u << WL) - 1u;
     const int inst = a.first_instance + blockIdx.x;
+    const unsigned thr_hi = a.hazard_thr >> 16, thr_lo = a.hazard_thr & 0xFFFFu;
 
     // ---- shared-memory carve-up (sizes match step_smem_bytes) ----
     int *q_key = reinterpret_cast<int *>(smem_raw);                                 // [W]
-    unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_key + W);    // [G][OW]
+    unsigned *q_id = reinterpret_cast<unsigned *>(q_key + W);                       // [W]
+    unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_id + W);     // [G][OW]
     unsigned *Lh_s = reinterpret_cast<unsigned *>(occ + (size_t)G * OW);            // [G][H1]
-    unsigned *load_new = Lh_s + (size_t)G * H1;                                     // [G]
-    int *nact_new = reinterpret_cast<int *>(load_new + G);                          // [G]
-    unsigned char *term_nib = reinterpret_cast<unsigned char *>(nact_new + G);      // [A/4]
-    int *scal = reinterpret_cast<int *>(term_nib + (((size_t)A / 4 + 15) & ~(size_t)15));
+    unsigned *sub_load = Lh_s + (size_t)G * H1;                                     // [G]
+    unsigned char *fin_b = reinterpret_cast<unsigned char *>(sub_load + G);         // [A/8]
+    unsigned char *eq_b = fin_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
+    int *scal = reinterpret_cast<int *>(eq_b + (((size_t)A8 + 15) & ~(size_t)15));
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue
 
@@ -144,19 +167,21 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
     if (n_w < 0 || n_w > W) { prologue_status |= BR_ST_BAD_STATE; n_w = n_w < 0 ? 0 : W; }
 
     if (tid < 16) scal[tid] = 0;
-    // queue -> packed keys in shared memory (16-byte loads)
+    // queue -> packed keys and ids in shared memory (16-byte loads)
     for (int i = tid * 4; i < n_w; i += NT * 4) {
         const int4 v = *reinterpret_cast<const int4 *>(g_qs + i);
+        const uint4 u = *reinterpret_cast<const uint4 *>(g_qid + i);
         int4 kk;
         kk.x = (v.x << WL) | (int)(posmask - (unsigned)(i + 0));
         kk.y = (v.y << WL) | (int)(posmask - (unsigned)(i + 1));
         kk.z = (v.z << WL) | (int)(posmask - (unsigned)(i + 2));
         kk.w = (v.w << WL) | (int)(posmask - (unsigned)(i + 3));
         *reinterpret_cast<int4 *>(q_key + i) = kk;
+        *reinterpret_cast<uint4 *>(q_id + i) = u;
     }
     for (int i = tid; i < G * OW; i += NT) occ[i] = g_occ[i];
     for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
-    for (int i = tid; i < G; i += NT) { load_new[i] = 0u; nact_new[i] = 0; }
+    for (int i = tid; i < G; i += NT) sub_load[i] = 0u;
 
     // router registers: lane owns workers lane and lane + 32
     int cap[GW];
@@ -180,6 +205,31 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
     __syncthreads();
     if (prologue_status) atomicOr(&scal[5], prologue_status);
 
+    // Philox words of the step's constant-hazard terminations: per 8-slot group one byte of
+    // "first 16 bits below the high half of the threshold" and one of "equal to it"
+    auto draw_terms = [&](int first, int stride) {
+#pragma unroll 1
+        for (int q8 = first; q8 < A8; q8 += stride) {
+            const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q8, kStreamTerm, 0u, key0, key1);
+            unsigned fb = 0, eb = 0;
+            const bool quick_ok = thr_hi < 0x8000u;
+            const unsigned any = quick_ok ? (hasless16(r.x, thr_hi + 1) | hasless16(r.y, thr_hi + 1) |
+                                             hasless16(r.z, thr_hi + 1) | hasless16(r.w, thr_hi + 1))
+                                          : 1u;
+            if (any) {
+                const unsigned wv[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const unsigned v = (wv[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
+                    fb |= (v < thr_hi ? 1u : 0u) << j;
+                    eb |= (v == thr_hi ? 1u : 0u) << j;
+                }
+            }
+            fin_b[q8] = (unsigned char)fb;
+            eq_b[q8] = (unsigned char)eb;
+        }
+    };
+
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + inst;
         const float *probs = a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr;
@@ -188,12 +238,22 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         if (timing) t_phase[0] = clock64();
 
         // ================= ARRIVE =================
+        // the arrival-count row is requested first; a single-warp block draws the termination
+        // words while that load is in flight
+        uint32_t row0 = 0xFFFFFFFFu, row1 = 0xFFFFFFFFu;
+        const uint32_t *row = nullptr;
+        if (a.arr_cdf) {
+            row = a.arr_cdf + ((size_t)inst * a.arr_inst_stride + (size_t)(k % a.arr_period)) * a.arr_len;
+            if (lane < a.arr_len) row0 = row[lane];
+            if (lane + 32 < a.arr_len) row1 = row[lane + 32];
+        }
+        if (nwarps == 1 && a.term_mode == 1) draw_terms(tid, NT);
         int n_arr = 0;
         if (a.arr_cdf) {
             const uint32_t u = philox4x32_10((uint32_t)k, 0u, kStreamArrCount, 0u, key0, key1).x;
-            const uint32_t *row = a.arr_cdf +
-                ((size_t)inst * a.arr_inst_stride + (size_t)(k % a.arr_period)) * a.arr_len;
-            for (int j0 = 0; j0 < a.arr_len; j0 += 32) {
+            n_arr = __popc(__ballot_sync(kFull, lane < a.arr_len && u >= row0)) +
+                    __popc(__ballot_sync(kFull, lane + 32 < a.arr_len && u >= row1));
+            for (int j0 = 64; j0 < a.arr_len; j0 += 32) {
                 const int j = j0 + lane;
                 const bool ge = (j < a.arr_len) && (u >= row[j]);
                 n_arr += __popc(__ballot_sync(kFull, ge));
@@ -208,6 +268,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                 const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)j >> 2, kStreamArrLen, 0u, key0, key1);
                 const int s = a.len_tab[word_of(r, j & 3) >> a.len_shift];
                 q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
+                q_id[pos] = id0 + (unsigned)j;
             }
         }
         int n_drop = n_w + n_arr - W;
@@ -219,6 +280,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         // ============ PREDICT (H > 0): c_hat maintenance + horizon projection ============
         if (H > 0) {
             const bool warp_uniform = (B % 32) == 0;
+#pragma unroll 1
             for (int s_base = 0; s_base < A; s_base += NT * kUnroll) {
                 int bs[kUnroll]; float c0s[kUnroll]; int krs[kUnroll];
 #pragma unroll
@@ -275,10 +337,21 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     }
                     const int g = (inr ? s0 : A - 1) / B;
                     if (warp_uniform) {
-                        for (int h = 0; h <= H; ++h) {
-                            const unsigned v = (live && h <= nh) ? (unsigned)(cur + h) : 0u;
-                            const unsigned s = __reduce_add_sync(kFull, v);
-                            if (lane == 0 && s) atomicAdd(&Lh_s[g * H1 + h], s);
+                        // common case: every running request of these 32 slots is counted at every
+                        // offset, so L_g(k+h) grows by (sum of loads) + h * (number of requests)
+                        const unsigned lv = __ballot_sync(kFull, live);
+                        const bool all_h = __all_sync(kFull, !live || nh == H);
+                        if (lv) {
+                            if (all_h) {
+                                const unsigned s = __reduce_add_sync(kFull, live ? (unsigned)cur : 0u);
+                                if (lane <= H) atomicAdd(&Lh_s[g * H1 + lane], s + (unsigned)(lane * __popc(lv)));
+                            } else {
+                                for (int h = 0; h <= H; ++h) {
+                                    const unsigned v = (live && h <= nh) ? (unsigned)(cur + h) : 0u;
+                                    const unsigned s = __reduce_add_sync(kFull, v);
+                                    if (lane == 0 && s) atomicAdd(&Lh_s[g * H1 + h], s);
+                                }
+                            }
                         }
                     } else if (live) {
                         for (int h = 0; h <= nh; ++h) atomicAdd(&Lh_s[g * H1 + h], (unsigned)(cur + h));
@@ -350,20 +423,38 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             // argmax_i F_g({i}) over all waiting requests, earliest arrival on ties.
             // Returns the packed key of the winner (0 if none).
             auto best_single = [&]() -> int {
-                long long bk = kNoKey; unsigned bt = 0; int bkey = 0;
-                for (int t = 0; t < n_tiles; ++t) {
-                    const int idx = (t << 5) + lane;
-                    const int qk = idx < n_w ? q_key[idx] : 0;
-                    if (qk > 0) {
-                        const long long f = sc.key(a, qk >> WL);
-                        const unsigned tie = (unsigned)qk & posmask;      // larger = earlier
-                        if (f > bk || (f == bk && tie > bt)) { bk = f; bt = tie; bkey = qk; }
+                if (!FP) {
+                    int bk = kEmpty; int bkey = 0;
+#pragma unroll 1
+                    for (int t = 0; t < n_tiles; ++t) {
+                        const int idx = (t << 5) + lane;
+                        const int qk = idx < n_w ? q_key[idx] : 0;
+                        if (qk > 0) {
+                            const int f = (int)sc.key(a, qk >> WL);
+                            // within a lane positions ascend, so strict > keeps the earliest
+                            if (f > bk) { bk = f; bkey = qk; }
+                        }
                     }
+                    int wk;
+                    const int src = warp_argmax_lane32(bk, (unsigned)bkey & posmask, wk);
+                    const int res = __shfl_sync(kFull, bkey, src);
+                    return res > 0 ? res : 0;
+                } else {
+                    long long bk = kNoKey; int bkey = 0;
+#pragma unroll 1
+                    for (int t = 0; t < n_tiles; ++t) {
+                        const int idx = (t << 5) + lane;
+                        const int qk = idx < n_w ? q_key[idx] : 0;
+                        if (qk > 0) {
+                            const long long f = sc.key(a, qk >> WL);
+                            if (f > bk) { bk = f; bkey = qk; }
+                        }
+                    }
+                    long long wk;
+                    const int src = warp_argmax_lane(bk, (unsigned)bkey & posmask, wk);
+                    const int res = __shfl_sync(kFull, bkey, src);
+                    return wk == kNoKey ? 0 : res;
                 }
-                long long wk;
-                const int src = warp_argmax_lane(bk, bt, wk);
-                const int res = __shfl_sync(kFull, bkey, src);
-                return wk == kNoKey ? 0 : res;
             };
 
             // sticky admission of the request with packed key qk to worker g
@@ -385,6 +476,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                             g_chat0[sa] = (float)(H + a.delta_T - 1);
                             g_kref[sa] = (uint8_t)((k + 1 - a.delta_T) & 255);
                         }
+                        if (g_aid) g_aid[sa] = q_id[pos];
                         q_key[pos] = (int)(0x80000000u | (unsigned)sa);
                     } else {
                         status |= BR_ST_BAD_STATE;
@@ -415,6 +507,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
 
             if (S_tot > 0 && n_w > 0) {
                 // ---------- Stage 1: greedy fill ----------
+#pragma unroll 1
                 while (S_tot > a.S_greedy && n_left > 0) {
                     if (s1_iters >= W) { status |= BR_ST_ITER_CAP; break; }
                     ++s1_iters;
@@ -436,6 +529,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             if (timing) t_phase[3] = clock64();
             if (S_tot > 0 && n_left > 0) {
                 // ---------- Stage 2: refined allocation ----------
+#pragma unroll 1
                 while (n_left > 0 && S_tot > 0) {
                     if (s2_pops >= W + G) { status |= BR_ST_ITER_CAP; break; }
                     ++s2_pops;
@@ -455,23 +549,30 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     const int g = (int)mg;
                     load_margins(g);
 
-                    // window: the R_max largest waiting requests, earliest first on ties
+                    // window: the R_max largest waiting requests, earliest first on ties.
+                    // One pass keeps each lane's four largest keys sorted; the heads are merged.
+                    int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0;
+#pragma unroll 1
+                    for (int t = 0; t < n_tiles; ++t) {
+                        const int idx = (t << 5) + lane;
+                        int x = idx < n_w ? q_key[idx] : 0;
+                        int y;
+                        y = max(t0, x); x = min(t0, x); t0 = y;
+                        y = max(t1, x); x = min(t1, x); t1 = y;
+                        y = max(t2, x); x = min(t2, x); t2 = y;
+                        y = max(t3, x); x = min(t3, x); t3 = y;
+                        t4 = max(t4, x);
+                    }
                     int win[BR_MAX_RMAX];
                     int nwin = 0;
-                    int prev = 0x7FFFFFFF;
 #pragma unroll
                     for (int r = 0; r < BR_MAX_RMAX; ++r) {
                         win[r] = 0;
                         if (r < a.R_max && r < n_left) {
-                            int best = 0;
-                            for (int t = 0; t < n_tiles; ++t) {
-                                const int idx = (t << 5) + lane;
-                                const int qk = idx < n_w ? q_key[idx] : 0;
-                                if (qk < prev && qk > best) best = qk;
-                            }
-                            best = __reduce_max_sync(kFull, best);
-                            win[r] = best; prev = best;
-                            if (best > 0) nwin = r + 1;
+                            const int m = __reduce_max_sync(kFull, t0);
+                            win[r] = m;
+                            if (m > 0) nwin = r + 1;
+                            if (t0 == m) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = 0; }
                         }
                     }
                     // subsets of the window: lane = mask, lowest mask on ties
@@ -527,41 +628,32 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             }
         } else if (a.term_mode == 1) {
             // warps 1.. draw this step's termination words while warp 0 routes
-            const int A4 = A >> 2;
-            for (int q4 = tid - 32; q4 < A4; q4 += NT - 32) {
-                const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
-                term_nib[q4] = (unsigned char)((r.x < a.hazard_thr ? 1 : 0) | (r.y < a.hazard_thr ? 2 : 0) |
-                                               (r.z < a.hazard_thr ? 4 : 0) | (r.w < a.hazard_thr ? 8 : 0));
-            }
+            draw_terms(tid - 32, NT - 32);
         }
         __syncthreads();                                              // B2: admissions visible
 
-        // ============ queue compaction, assignments, ids of admitted requests (warp 0) ============
+        // ============ queue compaction and assignments (warp 0) ============
         if (warp == 0) {
             int32_t *assign = a.assign_out + orow * W;
             int run = 0;
             const int n_before = n_w;          // queue length after ARRIVE
+#pragma unroll 1
             for (int i0 = 0; i0 < W; i0 += 32) {
                 const int i = i0 + lane;
                 const bool inq = i < n_before;
                 const int qk = inq ? q_key[i] : 0;
+                const unsigned id = inq ? q_id[i] : 0u;
                 const bool gone = inq && qk < 0;
                 const bool keep = inq && qk > 0;
                 const unsigned bal = __ballot_sync(kFull, keep);
                 const int dst = run + __popc(bal & ((1u << lane) - 1u));
                 const int sa = qk & 0x7FFFFFFF;
                 if (i < W) assign[i] = (gone && sa < A) ? sa : -1;
-                unsigned id = 0;
-                const bool fresh = i >= n_w_old;                  // arrived this step
-                const bool moved = keep && (dst != i || fresh);
-                if (!fresh && ((gone && g_aid) || moved)) id = g_qid[i];
-                if (fresh) id = id0 + (unsigned)(i - n_w_old);
                 __syncwarp();
-                if (gone && g_aid && sa < A) g_aid[sa] = id;
                 if (keep) {
                     const int s = qk >> WL;
-                    q_key[dst] = (s << WL) | (int)(posmask - (unsigned)dst);
-                    if (moved) { g_qs[dst] = s; g_qid[dst] = id; }
+                    if (dst != i) { q_key[dst] = (s << WL) | (int)(posmask - (unsigned)dst); q_id[dst] = id; }
+                    if (dst != i || i >= n_w_old) { g_qs[dst] = s; g_qid[dst] = id; }
                 }
                 __syncwarp();
                 run += __popc(bal);
@@ -576,81 +668,67 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         if (timing) t_phase[5] = clock64();
 
         // ================= ADVANCE (all warps) =================
-        {
-            const int A4 = A >> 2;
-            const bool pre = (nwarps > 1) && a.term_mode == 1;
-            for (int q_base = 0; q_base < A4; q_base += NT * kUnroll) {
-                int4 bv[kUnroll];
-#pragma unroll
-                for (int u = 0; u < kUnroll; ++u) {
-                    const int q4 = q_base + u * NT + tid;
-                    bv[u] = make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
-                    if (q4 < A4) bv[u] = *reinterpret_cast<const int4 *>(g_base + q4 * 4);
+        // occupancy byte & termination byte per 8-slot group; only slots whose request ends
+        // are read (to subtract their load) and written (freed)
+#pragma unroll 1
+        for (int q8 = tid; q8 < A8; q8 += NT) {
+            const int a0 = q8 << 3;
+            const int g = a0 / B, slot0 = a0 - g * B;
+            const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
+            if (!ob) continue;
+            unsigned ended = 0;
+            if (a.term_mode == 1) {
+                const unsigned fb = fin_b[q8], eb = eq_b[q8];
+                ended = ob & fb;
+                unsigned cand = ob & eb & ~fb;
+                while (cand) {                                       // first 16 bits tied: 16 more decide
+                    const int j = __ffs(cand) - 1;
+                    cand &= cand - 1;
+                    const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(a0 + j), kStreamTermRefine, 0u, key0, key1).x;
+                    if ((w & 0xFFFFu) < thr_lo) ended |= 1u << j;
                 }
+            } else if (a.term_mode == 2) {
+                const float sc24 = 5.9604644775390625e-8f;
 #pragma unroll
-                for (int u = 0; u < kUnroll; ++u) {
-                    if (q_base + u * NT >= A4) break;              // uniform across the block
-                    const int q4 = q_base + u * NT + tid;
-                    const bool inr = q4 < A4;
-                    const int4 b = bv[u];
-                    const bool any = (b.x != kEmpty) | (b.y != kEmpty) | (b.z != kEmpty) | (b.w != kEmpty);
-                    unsigned part = 0, ended = 0; int cnt = 0;
-                    if (any) {
-                        unsigned fin = 0;
-                        if (a.term_mode == 1) {
-                            if (pre) {
-                                fin = term_nib[q4];
-                            } else {
-                                const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
-                                fin = (r.x < a.hazard_thr ? 1u : 0u) | (r.y < a.hazard_thr ? 2u : 0u) |
-                                      (r.z < a.hazard_thr ? 4u : 0u) | (r.w < a.hazard_thr ? 8u : 0u);
-                            }
-                        } else if (a.term_mode == 2) {
-                            const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q4, kStreamTerm, 0u, key0, key1);
-                            const float *q = probs + (size_t)q4 * 4 * H;
-                            const float sc24 = 5.9604644775390625e-8f;
-                            fin = (__fmul_rn((float)(r.x >> 8), sc24) < q[0] ? 1u : 0u) |
-                                  (__fmul_rn((float)(r.y >> 8), sc24) < q[H] ? 2u : 0u) |
-                                  (__fmul_rn((float)(r.z >> 8), sc24) < q[2 * H] ? 4u : 0u) |
-                                  (__fmul_rn((float)(r.w >> 8), sc24) < q[3 * H] ? 8u : 0u);
-                        }
-                        int bb[4] = {b.x, b.y, b.z, b.w};
+                for (int half = 0; half < 2; ++half) {
+                    if (!((ob >> (4 * half)) & 0xFu)) continue;
+                    const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)(q8 * 2 + half), kStreamTerm, 0u, key0, key1);
+                    const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if (bb[j] == kEmpty) continue;
-                            if ((fin >> j) & 1u) { ended |= 1u << j; bb[j] = kEmpty; }
-                            else { part += (unsigned)(bb[j] + k + 1); cnt += 1; }
+                    for (int j = 0; j < 4; ++j) {
+                        const int jj = 4 * half + j;
+                        if ((ob >> jj) & 1u) {
+                            const float q = probs[(size_t)(a0 + jj) * H];
+                            if (__fmul_rn((float)(rr[j] >> 8), sc24) < q) ended |= 1u << jj;
                         }
-                        if (ended) *reinterpret_cast<int4 *>(g_base + q4 * 4) = make_int4(bb[0], bb[1], bb[2], bb[3]);
-                    }
-                    const int g = (inr ? q4 * 4 : A - 4) / B;
-                    // segmented sums over the lanes that hold the same worker
-                    unsigned peers;
-                    if ((B & 127) == 0) peers = kFull;
-                    else if (B == 64) peers = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
-                    else peers = __match_any_sync(kFull, g);
-                    const unsigned psum = __reduce_add_sync(peers, part);
-                    const int pcnt = (int)__reduce_add_sync(peers, (unsigned)cnt);
-                    if (lane == __ffs(peers) - 1 && inr && pcnt) {
-                        atomicAdd(&load_new[g], psum);
-                        atomicAdd(&nact_new[g], pcnt);
-                    }
-                    if (ended) {
-                        const int slot0 = (q4 * 4) % B;
-                        atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
                     }
                 }
+            }
+            if (ended) {
+                unsigned e = ended; unsigned sub = 0;
+                while (e) {
+                    const int j = __ffs(e) - 1;
+                    e &= e - 1;
+                    sub += (unsigned)(g_base[a0 + j] + k);
+                    g_base[a0 + j] = kEmpty;
+                }
+                atomicAdd(&sub_load[g], sub);
+                atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
             }
         }
         __syncthreads();                                              // B3
 
         if (warp == 0) {
+            // L_g(k+1) = L_g(k) - (loads of the requests that ended) + (number of survivors)
 #pragma unroll
             for (int w = 0; w < GW; ++w) {
                 const int g = lane + 32 * w;
                 if (g < G) {
-                    cap[w] = B - nact_new[g];
-                    L[w][0] = (int)load_new[g];
+                    int na = 0;
+                    for (int x = 0; x < OW; ++x) na += __popcll(occ[g * OW + x]);
+                    cap[w] = B - na;
+                    L[w][0] = L[w][0] - (int)sub_load[g] + na;
+                    sub_load[g] = 0u;
                 }
             }
             if (lane == 0) {
@@ -665,10 +743,6 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
 #pragma unroll
                     for (int p = 0; p < 6; ++p) pc[p] = (uint32_t)(t_phase[p + 1] - t_phase[p]);
                 }
-            }
-            __syncwarp();
-            if (it + 1 < a.n_steps) {
-                for (int i = lane; i < G; i += 32) { load_new[i] = 0u; nact_new[i] = 0; }
             }
         }
         if (it + 1 < a.n_steps) {

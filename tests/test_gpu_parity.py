@@ -78,8 +78,9 @@ def test_multi_step_launch_and_graph_replay():
 
 
 def test_ragged_shapes():
-    # G not a multiple of anything, B = 12 (not a multiple of 32), tiny and odd queue capacities
-    for G, B, W, H in [(1, 4, 4, 0), (3, 12, 20, 0), (5, 12, 36, 3), (7, 36, 100, 2), (64, 8, 64, 16)]:
+    # odd worker counts, B not a multiple of 32 or 64, tiny, odd and maximal queue capacities
+    for G, B, W, H in [(1, 8, 4, 0), (3, 24, 20, 0), (5, 16, 36, 3), (7, 40, 100, 2), (64, 8, 64, 16),
+                       (33, 72, 200, 5), (2, 256, 4096, 1)]:
         cfg = wlm.get_config("c0", G=G, B=B, W=W, H=H, init_active=B // 2, init_queue=W // 2,
                              hazard=0.05, term_mode=1, arrival=("const", 3.0), S_greedy=-1,
                              score_mode=-1, delta_T=-1, gate=0.1)

@@ -536,3 +536,18 @@ def test_stored_traces_are_reproduced():
         want = [tuple(int(x) for x in l.split()) for l in open(os.path.join(GOLDEN, f"{name}_trace.txt"))
                 if not l.startswith("#")]
         assert mg.run(name, steps) == want
+
+
+def test_hazard_decision_has_probability_thr_over_2_32():
+    """The 16 + 16 bit termination recipe fires exactly when the 32-bit word (v << 16 | w) is
+    below the threshold, so its probability is thr / 2^32."""
+    rng = np.random.default_rng(41)
+    for thr in [0, 1, 0xFFFF, 0x10000, wlm.hazard_threshold(1 / 500), wlm.hazard_threshold(1 / 400),
+                0x7FFF8001, 0xFFFFFFFF]:
+        hi = thr >> 16
+        vs = sorted(set([0, 1, max(hi - 1, 0), hi, min(hi + 1, 0xFFFF), 0xFFFF] + [int(x) for x in rng.integers(0, 65536, 20)]))
+        ws = [0, 1, (thr & 0xFFFF), max((thr & 0xFFFF) - 1, 0), min((thr & 0xFFFF) + 1, 0xFFFF), 0xFFFF] + \
+             [int(x) for x in rng.integers(0, 65536, 20)]
+        for v in vs:
+            for w in ws:
+                assert oracle.term_decision(v, w, thr) == (((v << 16) | w) < thr)
