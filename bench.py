@@ -170,7 +170,7 @@ def run_reference(args):
 class RotatingSets:
     """R independent instance sets of one configuration, stepped in rotation."""
 
-    def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=0):
+    def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=0, **params):
         import torch
         from paper_2605_06113_b200.binding import Router
         self.torch = torch
@@ -182,7 +182,7 @@ class RotatingSets:
             wl = wlm.make_workload(self.cfg, n_instances=n_inst, first_instance=seed_offset + r * n_inst)
             if self.router is None:
                 self.wl0 = wl
-                self.router = Router(wl, device=device, threads=threads)
+                self.router = Router(wl, device=device, threads=threads, **params)
                 arr_rows = [wl.arr_cdf]
             elif wl.arr_inst_stride:
                 arr_rows.append(wl.arr_cdf)
@@ -198,7 +198,7 @@ class RotatingSets:
                                    arr_cdf=table, arr_period=big.arr_period,
                                    arr_inst_stride=big.arr_inst_stride, hazard_thr=big.hazard_thr,
                                    state=big.state)
-            self.router = Router(big_tab, device=device, threads=threads)
+            self.router = Router(big_tab, device=device, threads=threads, **params)
         # all sets share one allocation per array so that `first_instance` selects the set
         keys = list(self.sets[0]["wl"].state.keys())
         cat = {k: np.concatenate([s["wl"].state[k] for s in self.sets], axis=0) for k in keys}

@@ -80,6 +80,7 @@ typedef struct {
     int32_t burst_every, burst_size; /* burst_size extra arrivals when k > 0 and k % burst_every == 0 */
     int32_t s_max;          /* largest prompt length the caller will ever enqueue (range proof) */
     int32_t threads;        /* threads per instance (multiple of 32, <= 256); <= 0 -> chosen from G*B, H and the batch size */
+    int32_t inst_per_block; /* instances per thread block when an instance runs on one warp (1..8); <= 0 -> 4 */
 } br_params;
 
 /* running requests; instance i occupies row first_instance + i of every array */
@@ -122,10 +123,11 @@ typedef struct {
                                      Stage-2 pops; may be NULL                                  */
     double   *fscore;     /* [N][W][G] optional: F_g({i}) of every waiting request before the
                                      first admission (0 beyond the queue length); NULL in timed runs */
-    uint32_t *phase_cycles; /* [N][6] optional: SM clock cycles this step spent in ARRIVE, PREDICT,
+    uint32_t *phase_cycles; /* [N][8] optional: SM clock cycles this step spent in ARRIVE, PREDICT,
                                      Stage 1, Stage 2, RECORD + queue compaction, ADVANCE (the split the
-                                     paper reports for its dispatcher: preparation / Stage 1 / Stage 2);
-                                     may be NULL */
+                                     paper reports for its dispatcher: preparation / Stage 1 / Stage 2),
+                                     then the launch's state-load prologue and its total from kernel
+                                     entry to the state write-back; may be NULL */
 } br_load_out;
 
 /*

@@ -28,7 +28,7 @@ class BrParams(C.Structure):
         ("arr_inst_stride", C.c_int32),
         ("len_tab", C.c_void_p), ("len_tab_log2", C.c_int32),
         ("burst_every", C.c_int32), ("burst_size", C.c_int32),
-        ("s_max", C.c_int32), ("threads", C.c_int32),
+        ("s_max", C.c_int32), ("threads", C.c_int32), ("inst_per_block", C.c_int32),
     ]
 
 

@@ -18,6 +18,7 @@ struct br_ctx {
     StepArgs base;            // constant part of the kernel arguments
     int threads;              // threads per instance for large batches
     int threads_small;        // ... for batches of a few instances (latency path)
+    int inst_per_block;       // single-warp instances per thread block
     size_t smem;
     // latency path
     cudaGraph_t graph;
@@ -99,8 +100,15 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.out = *out;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G);
     // few instances: the launch is latency-bound, so spread each instance over more warps
-    const int threads = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
-    kern<<<b->n_instances, threads, ctx->smem, stream>>>(a);
+    const int tpi = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
+    // single-warp instances are packed several to a block
+    int per_block = (tpi == 32) ? ctx->inst_per_block : 1;
+    if (per_block > b->n_instances) per_block = b->n_instances;
+    while (per_block > 1 && ctx->smem * per_block > 48 * 1024) --per_block;
+    a.tpi = tpi;
+    a.smem_per_inst = (int32_t)ctx->smem;
+    const int blocks = (b->n_instances + per_block - 1) / per_block;
+    kern<<<blocks, tpi * per_block, ctx->smem * per_block, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
     return BR_OK;
@@ -180,6 +188,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     memset(ctx, 0, sizeof(*ctx));
     ctx->G = G; ctx->H = H; ctx->p = p;
     ctx->threads = threads_large; ctx->threads_small = threads_small;
+    ctx->inst_per_block = p.inst_per_block > 0 ? (p.inst_per_block > 8 ? 8 : p.inst_per_block) : 4;
     StepArgs &a = ctx->base;
     a.G = G; a.H = H; a.B = p.B; a.W = p.W; a.R_max = p.R_max; a.S_greedy = p.S_greedy;
     a.occ_words = (p.B + 63) / 64;
@@ -294,7 +303,7 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
         {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
         {hout->fscore ? N * W * G * 8 : 0, (void **)&dout.fscore, hout->fscore, false, true},
-        {hout->phase_cycles ? N * 24 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
+        {hout->phase_cycles ? N * 32 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
     };
     size_t total = 0;
     for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;

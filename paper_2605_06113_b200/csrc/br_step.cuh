@@ -35,6 +35,7 @@ struct StepArgs {
     double aD, beta;
     double d[BR_MAX_H + 1];
     int32_t N, first_instance, n_steps;
+    int32_t tpi, smem_per_inst;  // threads and shared-memory bytes per instance
     br_worker_state ws;
     br_waiting_queue wq;
     const float *term_probs;
@@ -50,8 +51,8 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     n += 8 * (size_t)G * occ_words;              // occ
     n += 4 * (size_t)G * (H + 1);                // Lh_s (PREDICT accumulators)
     n += 4 * (size_t)G;                          // sub_load
-    n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
-    n += 64;                                     // scalars
+    n += 3 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b, pre_b
+    n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
     return (n + 15) & ~(size_t)15;
 }
 
@@ -121,19 +122,28 @@ __device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
 }
 
 constexpr int kUnroll = 4;      // loads in flight per thread in the BR-H streaming phase
+constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
 template <bool FP, int HM, int GW>
-__global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
+__global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const StepArgs a)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    extern __shared__ __align__(16) unsigned char smem_all[];
+    // a.tpi threads serve one instance; a block holds blockDim.x / a.tpi instances (more than one
+    // only when tpi == 32, so that an instance-wide barrier is a warp barrier)
+    const int NT = a.tpi;
+    const int tid = threadIdx.x % NT, lane = tid & 31, warp = tid >> 5;
+    const int in_block = threadIdx.x / NT, per_block = blockDim.x / NT;
+    if (blockIdx.x * per_block + in_block >= a.N) return;            // whole instance groups only
+    unsigned char *smem_raw = smem_all + (size_t)in_block * a.smem_per_inst;
+    auto inst_sync = [&]() { if (NT == 32) __syncwarp(); else __syncthreads(); };
     const int nwarps = NT >> 5;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
     const int A8 = A >> 3;
     const int WL = a.wl;
     const unsigned posmask = (1u << WL) - 1u;
-    const int inst = a.first_instance + blockIdx.x;
+    const int inst = a.first_instance + blockIdx.x * per_block + in_block;
     const unsigned thr_hi = a.hazard_thr >> 16, thr_lo = a.hazard_thr & 0xFFFFu;
+    const unsigned t_entry = (unsigned)clock64();
 
     // ---- shared-memory carve-up (sizes match step_smem_bytes) ----
     int *q_key = reinterpret_cast<int *>(smem_raw);                                 // [W]
@@ -143,9 +153,13 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
     unsigned *sub_load = Lh_s + (size_t)G * H1;                                     // [G]
     unsigned char *fin_b = reinterpret_cast<unsigned char *>(sub_load + G);         // [A/8]
     unsigned char *eq_b = fin_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
-    int *scal = reinterpret_cast<int *>(eq_b + (((size_t)A8 + 15) & ~(size_t)15));
+    unsigned char *pre_b = eq_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
+    unsigned short *end_list = reinterpret_cast<unsigned short *>(pre_b + (((size_t)A8 + 15) & ~(size_t)15));  // [kEndList]
+    unsigned short *pre_list = end_list + kEndList;                                 // [32]
+    int *scal = reinterpret_cast<int *>(pre_list + 32);
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
-    //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue
+    //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
+    //       [6] requests that ended this step and were not prefetched, [7] prefetched ones
 
     // ---- per-instance global rows ----
     long long *g_load = reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G;
@@ -167,8 +181,9 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
     if (n_w < 0 || n_w > W) { prologue_status |= BR_ST_BAD_STATE; n_w = n_w < 0 ? 0 : W; }
 
     if (tid < 16) scal[tid] = 0;
-    // queue -> packed keys and ids in shared memory (16-byte loads)
-    for (int i = tid * 4; i < n_w; i += NT * 4) {
+    // queue -> packed keys and ids in shared memory (16-byte loads).  The first chunks are
+    // requested without waiting for the queue length (rows always hold W entries).
+    auto fetch_queue = [&](int i) {
         const int4 v = *reinterpret_cast<const int4 *>(g_qs + i);
         const uint4 u = *reinterpret_cast<const uint4 *>(g_qid + i);
         int4 kk;
@@ -178,7 +193,13 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         kk.w = (v.w << WL) | (int)(posmask - (unsigned)(i + 3));
         *reinterpret_cast<int4 *>(q_key + i) = kk;
         *reinterpret_cast<uint4 *>(q_id + i) = u;
+    };
+    {
+        const int i0 = tid * 4, i1 = (NT + tid) * 4;
+        if (i0 < W) fetch_queue(i0);
+        if (i1 < W) fetch_queue(i1);
     }
+    for (int i = (2 * NT + tid) * 4; i < n_w; i += NT * 4) fetch_queue(i);
     for (int i = tid; i < G * OW; i += NT) occ[i] = g_occ[i];
     for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
     for (int i = tid; i < G; i += NT) sub_load[i] = 0u;
@@ -202,40 +223,47 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             L[w][0] = (int)g_load[g];
         }
     }
-    __syncthreads();
+    inst_sync();
     if (prologue_status) atomicOr(&scal[5], prologue_status);
 
     // Philox words of the step's constant-hazard terminations: per 8-slot group one byte of
     // "first 16 bits below the high half of the threshold" and one of "equal to it"
     auto draw_terms = [&](int first, int stride) {
 #pragma unroll 1
-        for (int q8 = first; q8 < A8; q8 += stride) {
-            const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)q8, kStreamTerm, 0u, key0, key1);
-            unsigned fb = 0, eb = 0;
-            const bool quick_ok = thr_hi < 0x8000u;
-            const unsigned any = quick_ok ? (hasless16(r.x, thr_hi + 1) | hasless16(r.y, thr_hi + 1) |
-                                             hasless16(r.z, thr_hi + 1) | hasless16(r.w, thr_hi + 1))
-                                          : 1u;
-            if (any) {
-                const unsigned wv[4] = {r.x, r.y, r.z, r.w};
+        for (int q_base = first; q_base < A8; q_base += 4 * stride) {
+            // four independent Philox blocks in flight per thread
+            uint4 r[4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const unsigned v = (wv[j >> 1] >> (16 * (j & 1))) & 0xFFFFu;
-                    fb |= (v < thr_hi ? 1u : 0u) << j;
-                    eb |= (v == thr_hi ? 1u : 0u) << j;
+            for (int u = 0; u < 4; ++u)
+                r[u] = philox4x32_10((uint32_t)k, (uint32_t)(q_base + u * stride), kStreamTerm, 0u, key0, key1);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int q8 = q_base + u * stride;
+                unsigned fb = 0, eb = 0;
+                const unsigned wv[4] = {r[u].x, r[u].y, r[u].z, r[u].w};
+                unsigned any = 1u;
+                if (thr_hi < 0x8000u)
+                    any = hasless16(wv[0], thr_hi + 1) | hasless16(wv[1], thr_hi + 1) |
+                          hasless16(wv[2], thr_hi + 1) | hasless16(wv[3], thr_hi + 1);
+                if (any) {          // rare: some 16-bit draw is at or below the high half of the threshold
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const unsigned lo16 = wv[w] & 0xFFFFu, hi16 = wv[w] >> 16;
+                        fb |= ((lo16 < thr_hi ? 1u : 0u) | (hi16 < thr_hi ? 2u : 0u)) << (2 * w);
+                        eb |= ((lo16 == thr_hi ? 1u : 0u) | (hi16 == thr_hi ? 2u : 0u)) << (2 * w);
+                    }
                 }
+                if (q8 < A8) { fin_b[q8] = (unsigned char)fb; eq_b[q8] = (unsigned char)eb; }
             }
-            fin_b[q8] = (unsigned char)fb;
-            eq_b[q8] = (unsigned char)eb;
         }
     };
 
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + inst;
         const float *probs = a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr;
-        long long t_phase[7];
+        unsigned t_phase[7];
         const bool timing = a.out.phase_cycles != nullptr && tid == 0;
-        if (timing) t_phase[0] = clock64();
+        if (timing) t_phase[0] = (unsigned)clock64();
 
         // ================= ARRIVE =================
         // the arrival-count row is requested first; a single-warp block draws the termination
@@ -247,7 +275,45 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             if (lane < a.arr_len) row0 = row[lane];
             if (lane + 32 < a.arr_len) row1 = row[lane + 32];
         }
-        if (nwarps == 1 && a.term_mode == 1) draw_terms(tid, NT);
+        // A single-warp instance also resolves, right away, which of the requests already
+        // running end at this step, and requests their loads: the values are used only after
+        // routing, so that memory latency is off the step's critical path.
+        const bool have_pre = (nwarps == 1 && a.term_mode == 1);
+        int pend = 0, n_pre = 0;
+        if (have_pre) {
+            draw_terms(tid, NT);
+            __syncwarp();
+#pragma unroll 1
+            for (int q8 = tid; q8 < A8; q8 += NT) {
+                const int a0 = q8 << 3;
+                const int g = a0 / B, slot0 = a0 - g * B;
+                const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
+                unsigned fb = fin_b[q8], eb = eq_b[q8];
+                unsigned cand = ob & eb & ~fb;
+                if (cand) {                                          // first 16 bits tied: 16 more decide
+                    eb &= ~cand;
+                    while (cand) {
+                        const int j = __ffs(cand) - 1;
+                        cand &= cand - 1;
+                        const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(a0 + j), kStreamTermRefine, 0u, key0, key1).x;
+                        if ((w & 0xFFFFu) < thr_lo) fb |= 1u << j;
+                    }
+                    fin_b[q8] = (unsigned char)fb;
+                    eq_b[q8] = (unsigned char)eb;
+                }
+                unsigned e = ob & fb, mark = 0;
+                while (e) {
+                    const int j = __ffs(e) - 1;
+                    e &= e - 1;
+                    const int at = atomicAdd(&scal[7], 1);
+                    if (at < 32) { pre_list[at] = (unsigned short)(a0 + j); mark |= 1u << j; }
+                }
+                pre_b[q8] = (unsigned char)mark;
+            }
+            __syncwarp();
+            n_pre = min(scal[7], 32);
+            if (tid < n_pre) pend = g_base[pre_list[tid]];
+        }
         int n_arr = 0;
         if (a.arr_cdf) {
             const uint32_t u = philox4x32_10((uint32_t)k, 0u, kStreamArrCount, 0u, key0, key1).x;
@@ -275,7 +341,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         n_drop = n_drop > 0 ? n_drop : 0;
         n_w = n_w + n_arr - n_drop;
         next_id += (uint32_t)n_arr;
-        if (timing) t_phase[1] = clock64();
+        if (timing) t_phase[1] = (unsigned)clock64();
 
         // ============ PREDICT (H > 0): c_hat maintenance + horizon projection ============
         if (H > 0) {
@@ -359,8 +425,8 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                 }
             }
         }
-        __syncthreads();                                              // B1
-        if (timing) t_phase[2] = clock64();
+        inst_sync();                                              // B1
+        if (timing) t_phase[2] = (unsigned)clock64();
 
         if (warp == 0) {
             // ================= ROUTE (warp 0 only, warp-synchronous) =================
@@ -425,7 +491,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             auto best_single = [&]() -> int {
                 if (!FP) {
                     int bk = kEmpty; int bkey = 0;
-#pragma unroll 1
+#pragma unroll 4
                     for (int t = 0; t < n_tiles; ++t) {
                         const int idx = (t << 5) + lane;
                         const int qk = idx < n_w ? q_key[idx] : 0;
@@ -526,7 +592,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     commit(qk, g);
                 }
             }
-            if (timing) t_phase[3] = clock64();
+            if (timing) t_phase[3] = (unsigned)clock64();
             if (S_tot > 0 && n_left > 0) {
                 // ---------- Stage 2: refined allocation ----------
 #pragma unroll 1
@@ -552,7 +618,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     // window: the R_max largest waiting requests, earliest first on ties.
                     // One pass keeps each lane's four largest keys sorted; the heads are merged.
                     int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0;
-#pragma unroll 1
+#pragma unroll 4
                     for (int t = 0; t < n_tiles; ++t) {
                         const int idx = (t << 5) + lane;
                         int x = idx < n_w ? q_key[idx] : 0;
@@ -600,7 +666,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     }
                 }
             }
-            if (timing) t_phase[4] = clock64();
+            if (timing) t_phase[4] = (unsigned)clock64();
 
             // ================= RECORD =================
             {
@@ -630,14 +696,14 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             // warps 1.. draw this step's termination words while warp 0 routes
             draw_terms(tid - 32, NT - 32);
         }
-        __syncthreads();                                              // B2: admissions visible
+        inst_sync();                                              // B2: admissions visible
 
         // ============ queue compaction and assignments (warp 0) ============
         if (warp == 0) {
             int32_t *assign = a.assign_out + orow * W;
             int run = 0;
             const int n_before = n_w;          // queue length after ARRIVE
-#pragma unroll 1
+#pragma unroll 2
             for (int i0 = 0; i0 < W; i0 += 32) {
                 const int i = i0 + lane;
                 const bool inq = i < n_before;
@@ -665,7 +731,7 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
             }
         }
         n_w = scal[0];
-        if (timing) t_phase[5] = clock64();
+        if (timing) t_phase[5] = (unsigned)clock64();
 
         // ================= ADVANCE (all warps) =================
         // occupancy byte & termination byte per 8-slot group; only slots whose request ends
@@ -705,18 +771,38 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                 }
             }
             if (ended) {
-                unsigned e = ended; unsigned sub = 0;
+                atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
+                unsigned e = have_pre ? (ended & ~(unsigned)pre_b[q8]) : ended;
                 while (e) {
                     const int j = __ffs(e) - 1;
                     e &= e - 1;
-                    sub += (unsigned)(g_base[a0 + j] + k);
-                    g_base[a0 + j] = kEmpty;
+                    const int at = atomicAdd(&scal[6], 1);
+                    if (at < kEndList) {
+                        end_list[at] = (unsigned short)(a0 + j);
+                    } else {                                   // list full: fix this slot up at once
+                        atomicAdd(&sub_load[g], (unsigned)(g_base[a0 + j] + k));
+                        g_base[a0 + j] = kEmpty;
+                    }
                 }
-                atomicAdd(&sub_load[g], sub);
-                atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
             }
         }
-        __syncthreads();                                              // B3
+        inst_sync();
+        {
+            // the requests that ended: subtract their load from the worker, free the slot
+            if (tid < n_pre) {
+                const int sa = pre_list[tid];
+                g_base[sa] = kEmpty;
+                atomicAdd(&sub_load[sa / B], (unsigned)(pend + k));
+            }
+            const int n_end = min(scal[6], kEndList);
+            for (int e = tid; e < n_end; e += NT) {
+                const int sa = end_list[e];
+                const int cur = g_base[sa] + k;
+                g_base[sa] = kEmpty;
+                atomicAdd(&sub_load[sa / B], (unsigned)cur);
+            }
+        }
+        inst_sync();                                              // B3
 
         if (warp == 0) {
             // L_g(k+1) = L_g(k) - (loads of the requests that ended) + (number of survivors)
@@ -737,17 +823,20 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
                     c[0] = (uint32_t)n_drop; c[1] = (uint32_t)scal[1]; c[2] = (uint32_t)scal[2]; c[3] = (uint32_t)scal[3];
                 }
                 if (a.out.status) a.out.status[orow] = scal[4] | scal[5];
+                scal[6] = 0; scal[7] = 0;
                 if (timing) {
-                    t_phase[6] = clock64();
-                    uint32_t *pc = a.out.phase_cycles + orow * 6;
+                    t_phase[6] = (unsigned)clock64();
+                    uint32_t *pc = a.out.phase_cycles + orow * 8;
 #pragma unroll
                     for (int p = 0; p < 6; ++p) pc[p] = (uint32_t)(t_phase[p + 1] - t_phase[p]);
+                    pc[6] = it == 0 ? (uint32_t)(t_phase[0] - t_entry) : 0u;
+                    pc[7] = 0u;
                 }
             }
         }
         if (it + 1 < a.n_steps) {
             for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
-            __syncthreads();
+            inst_sync();
         }
     }
 
@@ -764,6 +853,8 @@ __global__ void __launch_bounds__(256) br_step_kernel(const StepArgs a)
         a.ws.step[inst] = k;
         a.ws.next_id[inst] = next_id;
         a.wq.n[inst] = n_w;
+        if (a.out.phase_cycles)      // time from kernel entry to here, for the last step's row
+            a.out.phase_cycles[((size_t)(a.n_steps - 1) * a.N + inst) * 8 + 7] = (uint32_t)((unsigned)clock64() - t_entry);
     }
 }
 
