@@ -99,6 +99,23 @@ class ClockSampler:
         return out
 
 
+def shard_of(rank: int, world: int, instances_per_rank: int, sets: int = 1):
+    """First instance and instance count owned by `rank`: ranks own disjoint, equally sized
+    seed ranges (weak scaling); there is no exchange between ranks on the data path."""
+    n = instances_per_rank * sets
+    return rank * n, n
+
+
+def max_over_ranks(ms: float, dist, device="cuda") -> float:
+    """Timed region of the job = the slowest rank's."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def dist_setup(args):
     import torch
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -242,11 +259,9 @@ def time_launches(torch, fn, warmup, steps, dist=None):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
     if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = max_over_ranks(ms, dist)
         dist.barrier()
         torch.cuda.synchronize()
-        ms = float(t.item())
     return ms
 
 
@@ -299,7 +314,8 @@ def run_ours(args):
     N = cfg.N
     per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
     n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
-    sets = RotatingSets("c3", N, n_sets, device, seed_offset=rank * n_sets * N, threads=args.threads)
+    first, _ = shard_of(rank, world, N, n_sets)
+    sets = RotatingSets("c3", N, n_sets, device, seed_offset=first, threads=args.threads)
     sampler = ClockSampler(local)
     sampler.start()
     ms = time_launches(torch, sets.step, args.warmup, args.steps, dist)
@@ -337,9 +353,10 @@ def run_ours(args):
         except Exception as ex:  # keep the headline line even if an extra fails
             line["extra"] = {"error": repr(ex)}
         # ---------------- CPU baseline: the checker on host cores ----------------
-        rate, done, dt = oracle_rate("c3", 12.0, 16, 500)
+        rate, done, dt = oracle_rate("c3", 12.0, 64, 500)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{done} instance-steps of c3 (16 instances), {dt:.1f} s, single thread"}
+                                "sample": f"{done} instance-steps of c3 (first 64 instances, steps 0..{done // 64 - 1}), "
+                                          f"{dt:.1f} s, single thread"}
     elif rank == 0:
         line["e2e"] = None
     if rank == 0:
