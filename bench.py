@@ -233,13 +233,17 @@ class RotatingSets:
                 self.probs.append(wlm.term_probs_torch(self.wl0, j, device, seeds_t=seeds_t, tab_t=tab_t).contiguous())
         self.n_sets = n_sets
         self.launch = 0
+        self._calls = {}
 
     def step(self):
         r = self.launch % self.n_sets
-        probs = None
-        if self.probs is not None:
-            probs = self.probs[(self.launch // self.n_sets) % len(self.probs)]
-        self.router.step(self.st, self.out_view, probs, N=self.N, first=r * self.N)
+        j = (self.launch // self.n_sets) % len(self.probs) if self.probs is not None else 0
+        call = self._calls.get((r, j))
+        if call is None:       # argument marshalling is done once per (set, probability buffer)
+            probs = self.probs[j] if self.probs is not None else None
+            call = self.router.prepare(self.st, self.out_view, probs, N=self.N, first=r * self.N)
+            self._calls[(r, j)] = call
+        call()
         self.launch += 1
 
 

@@ -202,6 +202,21 @@ class Router:
         if rc != BR_OK:
             raise BrError(rc, "br_step")
 
+    def prepare(self, st, out, term_probs=None, N=None, first=0, n_steps=1, stream=None):
+        """Marshals the arguments of br_step once; the returned callable repeats the same call
+        (same buffers, same stream) without rebuilding the argument structures."""
+        N = st["step"].shape[0] - first if N is None else N
+        b, ws, wq, lo = self._structs(st, out, N, first, n_steps, self._stream(stream))
+        fn, h = lib().br_step, self._h
+        args = (h, C.byref(b), C.byref(ws), C.byref(wq), _ptr(term_probs), _ptr(out["assign"]), C.byref(lo))
+        keep = (b, ws, wq, lo, st, out, term_probs)
+
+        def call(_fn=fn, _args=args, _keep=keep):
+            rc = _fn(*_args)
+            if rc != BR_OK:
+                raise BrError(rc, "br_step")
+        return call
+
     def graph_capture(self, st, out, term_probs=None, N=None, first=0, n_steps=1, stream=None):
         N = st["step"].shape[0] - first if N is None else N
         b, ws, wq, lo = self._structs(st, out, N, first, n_steps, self._stream(stream))

@@ -48,10 +48,10 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
 {
     size_t n = 0;
     n += 4 * (size_t)W * 2;                      // q_key, q_id
-    n += 8 * (size_t)G * occ_words;              // occ
+    n += 8 * (size_t)G * occ_words * 2;          // occ, end_mask
     n += 4 * (size_t)G * (H + 1);                // Lh_s (PREDICT accumulators)
     n += 4 * (size_t)G;                          // sub_load
-    n += 3 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b, pre_b
+    n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
     return (n + 15) & ~(size_t)15;
 }
@@ -149,12 +149,12 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
     int *q_key = reinterpret_cast<int *>(smem_raw);                                 // [W]
     unsigned *q_id = reinterpret_cast<unsigned *>(q_key + W);                       // [W]
     unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_id + W);     // [G][OW]
-    unsigned *Lh_s = reinterpret_cast<unsigned *>(occ + (size_t)G * OW);            // [G][H1]
-    unsigned *sub_load = Lh_s + (size_t)G * H1;                                     // [G]
-    unsigned char *fin_b = reinterpret_cast<unsigned char *>(sub_load + G);         // [A/8]
+    unsigned long long *end_mask = occ + (size_t)G * OW;                            // [G][OW]
+    unsigned char *fin_b = reinterpret_cast<unsigned char *>(end_mask + (size_t)G * OW);   // [A/8], 8-byte aligned
     unsigned char *eq_b = fin_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
-    unsigned char *pre_b = eq_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
-    unsigned short *end_list = reinterpret_cast<unsigned short *>(pre_b + (((size_t)A8 + 15) & ~(size_t)15));  // [kEndList]
+    unsigned *Lh_s = reinterpret_cast<unsigned *>(eq_b + (((size_t)A8 + 15) & ~(size_t)15));   // [G][H1]
+    unsigned *sub_load = Lh_s + (size_t)G * H1;                                     // [G]
+    unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
     unsigned short *pre_list = end_list + kEndList;                                 // [32]
     int *scal = reinterpret_cast<int *>(pre_list + 32);
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
@@ -242,9 +242,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
                 unsigned fb = 0, eb = 0;
                 const unsigned wv[4] = {r[u].x, r[u].y, r[u].z, r[u].w};
                 unsigned any = 1u;
-                if (thr_hi < 0x8000u)
-                    any = hasless16(wv[0], thr_hi + 1) | hasless16(wv[1], thr_hi + 1) |
-                          hasless16(wv[2], thr_hi + 1) | hasless16(wv[3], thr_hi + 1);
+                if (thr_hi < 0x8000u)       // smallest 16-bit draw of the block against the threshold
+                    any = hasless16(__vminu2(__vminu2(wv[0], wv[1]), __vminu2(wv[2], wv[3])), thr_hi + 1);
                 if (any) {          // rare: some 16-bit draw is at or below the high half of the threshold
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
@@ -254,6 +253,58 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
                     }
                 }
                 if (q8 < A8) { fin_b[q8] = (unsigned char)fb; eq_b[q8] = (unsigned char)eb; }
+            }
+        }
+    };
+
+    // Per worker word: which running requests end at this step (occupancy & termination draws).
+    // Writes end_mask and lists the ending slots; with `prefetch` the first 32 go to pre_list so
+    // that their loads can be requested at once by one lane each.
+    auto scan_workers = [&](bool prefetch) {
+#pragma unroll 1
+        for (int idx = tid; idx < G * OW; idx += NT) {
+            const int g = idx / OW, x = idx - g * OW;
+            const unsigned long long occw = occ[idx];
+            unsigned long long finw = 0ull, eqw = 0ull;
+            if (a.term_mode != 0 && occw) {
+                const int b0 = g * (B >> 3) + 8 * x;
+                const int nb = min(8, (B >> 3) - 8 * x);
+                if (nb == 8 && (b0 & 7) == 0) {
+                    finw = *reinterpret_cast<const unsigned long long *>(fin_b + b0);
+                    eqw = *reinterpret_cast<const unsigned long long *>(eq_b + b0);
+                } else {
+                    for (int b = 0; b < nb; ++b) {
+                        finw |= (unsigned long long)fin_b[b0 + b] << (8 * b);
+                        eqw |= (unsigned long long)eq_b[b0 + b] << (8 * b);
+                    }
+                }
+                unsigned long long cand = occw & eqw & ~finw;
+                while (cand) {                                       // first 16 bits tied: 16 more decide
+                    const int j = __ffsll((long long)cand) - 1;
+                    cand &= cand - 1;
+                    const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(g * B + 64 * x + j),
+                                                     kStreamTermRefine, 0u, key0, key1).x;
+                    if ((w & 0xFFFFu) < thr_lo) finw |= 1ull << j;
+                }
+            }
+            unsigned long long ended = occw & finw;
+            end_mask[idx] = ended;
+            while (ended) {
+                const int j = __ffsll((long long)ended) - 1;
+                ended &= ended - 1;
+                const int sa = g * B + 64 * x + j;
+                int at = prefetch ? atomicAdd(&scal[7], 1) : 32;
+                if (at < 32) {
+                    pre_list[at] = (unsigned short)sa;
+                } else {
+                    at = atomicAdd(&scal[6], 1);
+                    if (at < kEndList) {
+                        end_list[at] = (unsigned short)sa;
+                    } else {                                         // list full: fix this slot up at once
+                        atomicAdd(&sub_load[g], (unsigned)(g_base[sa] + k));
+                        g_base[sa] = kEmpty;
+                    }
+                }
             }
         }
     };
@@ -283,33 +334,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
         if (have_pre) {
             draw_terms(tid, NT);
             __syncwarp();
-#pragma unroll 1
-            for (int q8 = tid; q8 < A8; q8 += NT) {
-                const int a0 = q8 << 3;
-                const int g = a0 / B, slot0 = a0 - g * B;
-                const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
-                unsigned fb = fin_b[q8], eb = eq_b[q8];
-                unsigned cand = ob & eb & ~fb;
-                if (cand) {                                          // first 16 bits tied: 16 more decide
-                    eb &= ~cand;
-                    while (cand) {
-                        const int j = __ffs(cand) - 1;
-                        cand &= cand - 1;
-                        const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(a0 + j), kStreamTermRefine, 0u, key0, key1).x;
-                        if ((w & 0xFFFFu) < thr_lo) fb |= 1u << j;
-                    }
-                    fin_b[q8] = (unsigned char)fb;
-                    eq_b[q8] = (unsigned char)eb;
-                }
-                unsigned e = ob & fb, mark = 0;
-                while (e) {
-                    const int j = __ffs(e) - 1;
-                    e &= e - 1;
-                    const int at = atomicAdd(&scal[7], 1);
-                    if (at < 32) { pre_list[at] = (unsigned short)(a0 + j); mark |= 1u << j; }
-                }
-                pre_b[q8] = (unsigned char)mark;
-            }
+            scan_workers(true);
             __syncwarp();
             n_pre = min(scal[7], 32);
             if (tid < n_pre) pend = g_base[pre_list[tid]];
@@ -715,6 +740,25 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
                 const int dst = run + __popc(bal & ((1u << lane) - 1u));
                 const int sa = qk & 0x7FFFFFFF;
                 if (i < W) assign[i] = (gone && sa < A) ? sa : -1;
+                if (have_pre && gone && sa < A) {
+                    // a request admitted at this step may also end at it
+                    unsigned fb = (fin_b[sa >> 3] >> (sa & 7)) & 1u;
+                    if (!fb && ((eq_b[sa >> 3] >> (sa & 7)) & 1u)) {
+                        const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)sa, kStreamTermRefine, 0u, key0, key1).x;
+                        fb = (w & 0xFFFFu) < thr_lo;
+                    }
+                    if (fb) {
+                        const int g = sa / B, slot = sa - g * B;
+                        atomicOr(&end_mask[g * OW + (slot >> 6)], 1ull << (slot & 63));
+                        const int at = atomicAdd(&scal[6], 1);
+                        if (at < kEndList) {
+                            end_list[at] = (unsigned short)sa;
+                        } else {
+                            atomicAdd(&sub_load[g], (unsigned)(g_base[sa] + k));
+                            g_base[sa] = kEmpty;
+                        }
+                    }
+                }
                 __syncwarp();
                 if (keep) {
                     const int s = qk >> WL;
@@ -733,58 +777,38 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
         n_w = scal[0];
         if (timing) t_phase[5] = (unsigned)clock64();
 
-        // ================= ADVANCE (all warps) =================
-        // occupancy byte & termination byte per 8-slot group; only slots whose request ends
-        // are read (to subtract their load) and written (freed)
-#pragma unroll 1
-        for (int q8 = tid; q8 < A8; q8 += NT) {
-            const int a0 = q8 << 3;
-            const int g = a0 / B, slot0 = a0 - g * B;
-            const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
-            if (!ob) continue;
-            unsigned ended = 0;
-            if (a.term_mode == 1) {
-                const unsigned fb = fin_b[q8], eb = eq_b[q8];
-                ended = ob & fb;
-                unsigned cand = ob & eb & ~fb;
-                while (cand) {                                       // first 16 bits tied: 16 more decide
-                    const int j = __ffs(cand) - 1;
-                    cand &= cand - 1;
-                    const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(a0 + j), kStreamTermRefine, 0u, key0, key1).x;
-                    if ((w & 0xFFFFu) < thr_lo) ended |= 1u << j;
-                }
-            } else if (a.term_mode == 2) {
+        // ================= ADVANCE =================
+        // Only the occupancy masks, the termination draws and the few ending slots are touched.
+        if (!have_pre) {
+            if (a.term_mode == 2) {
+                // Bernoulli(term_probs[slot][0]) per running request: 24-bit uniform below the probability
                 const float sc24 = 5.9604644775390625e-8f;
+#pragma unroll 1
+                for (int q8 = tid; q8 < A8; q8 += NT) {
+                    const int a0 = q8 << 3;
+                    const int g = a0 / B, slot0 = a0 - g * B;
+                    const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
+                    unsigned fb = 0;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    if (!((ob >> (4 * half)) & 0xFu)) continue;
-                    const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)(q8 * 2 + half), kStreamTerm, 0u, key0, key1);
-                    const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
+                    for (int half = 0; half < 2; ++half) {
+                        if (!((ob >> (4 * half)) & 0xFu)) continue;
+                        const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)(q8 * 2 + half), kStreamTerm, 0u, key0, key1);
+                        const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int jj = 4 * half + j;
-                        if ((ob >> jj) & 1u) {
-                            const float q = probs[(size_t)(a0 + jj) * H];
-                            if (__fmul_rn((float)(rr[j] >> 8), sc24) < q) ended |= 1u << jj;
+                        for (int j = 0; j < 4; ++j) {
+                            const int jj = 4 * half + j;
+                            if ((ob >> jj) & 1u) {
+                                const float q = probs[(size_t)(a0 + jj) * H];
+                                if (__fmul_rn((float)(rr[j] >> 8), sc24) < q) fb |= 1u << jj;
+                            }
                         }
                     }
+                    fin_b[q8] = (unsigned char)fb;
+                    eq_b[q8] = 0;
                 }
+                inst_sync();
             }
-            if (ended) {
-                atomicAnd(&occ[g * OW + (slot0 >> 6)], ~((unsigned long long)ended << (slot0 & 63)));
-                unsigned e = have_pre ? (ended & ~(unsigned)pre_b[q8]) : ended;
-                while (e) {
-                    const int j = __ffs(e) - 1;
-                    e &= e - 1;
-                    const int at = atomicAdd(&scal[6], 1);
-                    if (at < kEndList) {
-                        end_list[at] = (unsigned short)(a0 + j);
-                    } else {                                   // list full: fix this slot up at once
-                        atomicAdd(&sub_load[g], (unsigned)(g_base[a0 + j] + k));
-                        g_base[a0 + j] = kEmpty;
-                    }
-                }
-            }
+            scan_workers(false);
         }
         inst_sync();
         {
@@ -811,7 +835,11 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
                 const int g = lane + 32 * w;
                 if (g < G) {
                     int na = 0;
-                    for (int x = 0; x < OW; ++x) na += __popcll(occ[g * OW + x]);
+                    for (int x = 0; x < OW; ++x) {
+                        const unsigned long long o = occ[g * OW + x] & ~end_mask[g * OW + x];
+                        occ[g * OW + x] = o;
+                        na += __popcll(o);
+                    }
                     cap[w] = B - na;
                     L[w][0] = L[w][0] - (int)sub_load[g] + na;
                     sub_load[g] = 0u;
@@ -845,10 +873,13 @@ __global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const Step
 #pragma unroll
         for (int w = 0; w < GW; ++w) {
             const int g = lane + 32 * w;
-            if (g < G) { g_load[g] = (long long)L[w][0]; g_nact[g] = B - cap[w]; }
+            if (g < G) {
+                g_load[g] = (long long)L[w][0];
+                g_nact[g] = B - cap[w];
+                for (int x = 0; x < OW; ++x) g_occ[g * OW + x] = occ[g * OW + x];   // updated by this lane
+            }
         }
     }
-    for (int i = tid; i < G * OW; i += NT) g_occ[i] = occ[i];
     if (tid == 0) {
         a.ws.step[inst] = k;
         a.ws.next_id[inst] = next_id;
