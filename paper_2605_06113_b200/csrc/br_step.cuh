@@ -125,7 +125,7 @@ constexpr int kUnroll = 4;      // loads in flight per thread in the BR-H stream
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
 template <bool FP, int HM, int GW>
-__global__ void __maxnreg__((FP && HM > 0) ? 255 : 72) br_step_kernel(const StepArgs a)
+__global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const StepArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_all[];
     // a.tpi threads serve one instance; a block holds blockDim.x / a.tpi instances (more than one
