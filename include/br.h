@@ -37,6 +37,7 @@ extern "C" {
 #define BR_ECUDA    -3   /* a CUDA runtime call failed; br_strerror gives its text        */
 #define BR_ENOMEM   -4   /* host or device allocation failed (br_create, host-buffer path)*/
 #define BR_ESTATE   -5   /* call order violated (e.g. br_graph_step before capture)       */
+#define BR_ELIMIT   -6   /* br_step_host_static: the batch does not fit BR_STATIC_STAGE_BYTES */
 
 /* compiled limits */
 #define BR_MAX_G      64
@@ -177,6 +178,36 @@ int br_graph_step(br_ctx *ctx);
 int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
                  br_waiting_queue *waiting_queue, const float *term_probs, int32_t *assign_out,
                  br_load_out *load_out, int64_t *h2d_bytes, int64_t *d2h_bytes);
+
+/*
+ * br_step_host for callers that must not allocate.  (The paper has no counterpart: this entry
+ * point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unsafe -- inside a
+ * latency-critical serving loop whose memory is fully pre-planned, in a process whose CUDA
+ * memory pool is owned by another framework and sized to the last byte, or in a callback /
+ * signal-like context where cudaMalloc (which may synchronise the device and take driver
+ * locks) can stall or deadlock.  br_step_host grows a staging buffer with cudaMalloc on
+ * demand; this variant never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * The device-side staging is a fixed array of BR_STATIC_STAGE_BYTES built into the library
+ * image, so every GPU that loads the library holds that much memory until the process exits.
+ * A batch whose snapshot plus outputs (each array padded to 256 bytes) exceeds it is rejected
+ * with BR_ELIMIT before anything is copied; load_out->fscore must be NULL (BR_EINVAL).
+ * Otherwise arguments, results and status codes are those of br_step_host.
+ *
+ * The first call on each device looks up the array's device address (a CUDA runtime query
+ * made with that device current; no allocation).  Make that first call outside any stream
+ * capture.  All calls on a device share the one array, which still holds the previous
+ * call's data: inputs are overwritten by the copies of this call and the output blocks are
+ * cleared first, but two calls that overlap on the GPU (different streams, or different host
+ * threads) race on it -- serialise them.  The call returns after synchronising the stream.
+ */
+#define BR_STATIC_STAGE_BYTES (8u << 20)
+int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
+                        br_waiting_queue *waiting_queue, const float *term_probs,
+                        int32_t *assign_out, br_load_out *load_out, int64_t *h2d_bytes,
+                        int64_t *d2h_bytes);
 
 /*
  * F-score matrix alone (Eq. 1 / Eq. 2 for single requests): for n_requests prompt lengths s

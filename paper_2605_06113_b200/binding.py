@@ -13,7 +13,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libbr.so")
 
-BR_OK, BR_EINVAL, BR_ERANGE, BR_ECUDA, BR_ENOMEM, BR_ESTATE = 0, -1, -2, -3, -4, -5
+BR_OK, BR_EINVAL, BR_ERANGE, BR_ECUDA, BR_ENOMEM, BR_ESTATE, BR_ELIMIT = 0, -1, -2, -3, -4, -5, -6
+STATIC_STAGE_BYTES = 8 << 20
 ST_QUEUE_OVERFLOW, ST_ITER_CAP, ST_BAD_STATE = 1, 2, 4
 EMPTY = -(2 ** 31)
 
@@ -53,6 +54,7 @@ class BrLoadOut(C.Structure):
 
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
+           "br_step_host_static",
            "br_fscore", "br_destroy", "br_strerror", "br_version"]
 
 _lib = None
@@ -80,6 +82,7 @@ def lib():
         L.br_graph_capture.argtypes = step_args
         L.br_graph_step.argtypes = [C.c_void_p]
         L.br_step_host.argtypes = step_args + [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.br_step_host_static.argtypes = step_args + [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.br_fscore.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_destroy.argtypes = [C.c_void_p]
@@ -239,6 +242,18 @@ class Router:
                                 _ptr(out["assign"]), C.byref(lo), C.byref(up), C.byref(down))
         if rc != BR_OK:
             raise BrError(rc, "br_step_host")
+        return up.value, down.value
+
+    def step_host_static(self, st, out, term_probs=None, N=None, stream=None):
+        """br_step_host_static: like step_host, but the device staging is the library's built-in
+        array, so nothing is allocated; raises BrError(BR_ELIMIT) if the batch does not fit."""
+        N = st["step"].shape[0] if N is None else N
+        b, ws, wq, lo = self._structs(st, out, N, 0, 1, self._stream(stream))
+        up, down = C.c_int64(), C.c_int64()
+        rc = lib().br_step_host_static(self._h, C.byref(b), C.byref(ws), C.byref(wq), _ptr(term_probs),
+                                       _ptr(out["assign"]), C.byref(lo), C.byref(up), C.byref(down))
+        if rc != BR_OK:
+            raise BrError(rc, "br_step_host_static")
         return up.value, down.value
 
     def fscore(self, s, Lh, F, cap=None, best_g=None, N=None, first=0, stream=None):

@@ -129,6 +129,7 @@ const char *br_strerror(int status)
     case BR_ECUDA: return g_cuda_msg;
     case BR_ENOMEM: return "allocation failed";
     case BR_ESTATE: return "call order violated";
+    case BR_ELIMIT: return "batch needs more staging than the built-in no-allocation buffer holds (BR_STATIC_STAGE_BYTES)";
     default: return "unknown status";
     }
 }
@@ -322,6 +323,116 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
     }
     br_instance_batch db = *batch; db.n_steps = 1;
     int rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
+    if (rc != BR_OK) return rc;
+    rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
+    if (rc != BR_OK) return rc;
+    for (Blk &b : blks) {
+        if (!b.bytes || !b.out) continue;
+        BR_CUDA(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, st));
+        down += (int64_t)b.bytes;
+    }
+    BR_CUDA(cudaStreamSynchronize(st));
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return BR_OK;
+}
+
+/* ---- host-buffer step without any allocation ------------------------------------------- */
+
+// Staging for br_step_host_static.  It lives in the library image: every GPU that loads the
+// library holds these bytes until the process exits, and every call on a device shares them.
+static __device__ __align__(256) unsigned char g_static_stage[BR_STATIC_STAGE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_stage_ptr[kMaxDevices];      // device address of g_static_stage, per device
+
+// In host code `g_static_stage` is only a handle; the address a kernel or a copy can use
+// has to be asked for, once per device, with that device current.
+int static_stage_address(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return BR_EINVAL;
+    if (!g_static_stage_ptr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_static_stage);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(g_static_stage)");
+        g_static_stage_ptr[dev] = ptr;
+    }
+    *out = g_static_stage_ptr[dev];
+    return BR_OK;
+}
+}  // namespace
+
+int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *hws,
+                        br_waiting_queue *hwq, const float *h_probs, int32_t *h_assign,
+                        br_load_out *hout, int64_t *h2d_bytes, int64_t *d2h_bytes)
+{
+    if (!ctx || !batch || !hws || !hwq || !hout) return BR_EINVAL;
+    if (batch->n_instances < 0 || batch->first_instance != 0 || batch->n_steps > 1) return BR_EINVAL;
+    if (!hws->load || !hws->nact || !hws->occ || !hws->act_base || !hws->step || !hws->seed ||
+        !hws->next_id || !hwq->s || !hwq->id || !hwq->n || !h_assign || !hout->load || !hout->trace)
+        return BR_EINVAL;
+    if (ctx->H > 0 && (!hws->act_chat0 || !hws->act_kref || !h_probs)) return BR_EINVAL;
+    if (ctx->p.term_mode == 2 && !h_probs) return BR_EINVAL;
+    if (hout->fscore) return BR_EINVAL;                 // the score matrix is not offered on this path
+    const size_t N = (size_t)batch->n_instances;
+    if (N == 0) return BR_OK;
+    const size_t G = ctx->G, H = ctx->H, B = ctx->p.B, W = ctx->p.W, A = G * B;
+    const size_t OW = (B + 63) / 64;
+    cudaStream_t st = (cudaStream_t)batch->stream;
+
+    struct Blk { size_t bytes; void **dev; void *host; bool in, out; };
+    br_worker_state dws; memset(&dws, 0, sizeof(dws));
+    br_waiting_queue dwq; memset(&dwq, 0, sizeof(dwq));
+    br_load_out dout; memset(&dout, 0, sizeof(dout));
+    float *d_probs = nullptr; int32_t *d_assign = nullptr;
+    const bool pred = H > 0;
+    Blk blks[] = {
+        {N * G * 8, (void **)&dws.load, hws->load, true, true},
+        {N * G * 4, (void **)&dws.nact, hws->nact, true, true},
+        {N * G * OW * 8, (void **)&dws.occ, hws->occ, true, true},
+        {N * A * 4, (void **)&dws.act_base, hws->act_base, true, true},
+        {hws->act_id ? N * A * 4 : 0, (void **)&dws.act_id, hws->act_id, true, true},
+        {pred ? N * A * 4 : 0, (void **)&dws.act_chat0, hws->act_chat0, true, true},
+        {pred ? N * A : 0, (void **)&dws.act_kref, hws->act_kref, true, true},
+        {N * 4, (void **)&dws.step, hws->step, true, true},
+        {N * 8, (void **)&dws.seed, hws->seed, true, false},
+        {N * 4, (void **)&dws.next_id, hws->next_id, true, true},
+        {N * W * 4, (void **)&dwq.s, hwq->s, true, true},
+        {N * W * 4, (void **)&dwq.id, hwq->id, true, true},
+        {N * 4, (void **)&dwq.n, hwq->n, true, true},
+        {h_probs ? N * A * H * 4 : 0, (void **)&d_probs, (void *)h_probs, true, false},
+        {N * W * 4, (void **)&d_assign, h_assign, false, true},
+        {N * G * 8, (void **)&dout.load, hout->load, false, true},
+        {N * 3 * 8, (void **)&dout.trace, hout->trace, false, true},
+        {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
+        {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
+        {hout->phase_cycles ? N * 32 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
+    };
+    size_t total = 0;
+    for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;
+    if (total > (size_t)BR_STATIC_STAGE_BYTES) return BR_ELIMIT;      // nothing was touched
+
+    void *stage = nullptr;
+    int rc = static_stage_address(&stage);
+    if (rc != BR_OK) return rc;
+
+    size_t off = 0, out_begin = 0, out_end = 0;
+    int64_t up = 0, down = 0;
+    for (Blk &b : blks) {
+        if (!b.bytes) continue;
+        *b.dev = (char *)stage + off;
+        if (!b.in) { if (!out_end) out_begin = off; out_end = off + ((b.bytes + 255) & ~(size_t)255); }
+        off += (b.bytes + 255) & ~(size_t)255;
+        if (b.in) { BR_CUDA(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, st)); up += (int64_t)b.bytes; }
+    }
+    // the buffer still holds the previous call's results: the output blocks start from zero
+    if (out_end > out_begin) BR_CUDA(cudaMemsetAsync((char *)stage + out_begin, 0, out_end - out_begin, st));
+    br_instance_batch db = *batch; db.n_steps = 1;
+    rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
     if (rc != BR_OK) return rc;
     rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
     if (rc != BR_OK) return rc;
