@@ -178,7 +178,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         threads_small = threads_large = p.threads;
     } else {
         const int work = A * (H > 0 ? 2 : 1);
-        int w = (work + 2047) / 2048;
+        int w = (work + 4095) / 4096;
         threads_large = 32 * (w < 1 ? 1 : (w > 8 ? 8 : w));
         w = (work + 1023) / 1024;
         threads_small = 32 * (w < 1 ? 1 : (w > 8 ? 8 : w));
@@ -194,6 +194,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     a.G = G; a.H = H; a.B = p.B; a.W = p.W; a.R_max = p.R_max; a.S_greedy = p.S_greedy;
     a.occ_words = (p.B + 63) / 64;
     a.wl = wl;
+    a.magic_B = (uint32_t)(((1ull << 32) + (unsigned)p.B - 1) / (unsigned)p.B);
     a.delta_T = p.delta_T; a.gate = p.gate; a.c_floor = p.c_floor;
     a.term_mode = p.term_mode; a.hazard_thr = p.hazard_thr;
     a.arr_cdf = p.arr_cdf; a.arr_len = p.arr_len; a.arr_period = p.arr_period;

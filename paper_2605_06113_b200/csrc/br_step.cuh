@@ -23,6 +23,7 @@ namespace br {
 struct StepArgs {
     int32_t G, H, B, W, R_max, S_greedy, occ_words;
     int32_t wl;                 // log2 of the queue-position field of a packed key
+    uint32_t magic_B;           // ceil(2^32 / B): x / B == umulhi(x, magic_B) for x < 2^16
     int32_t delta_T;
     float gate, c_floor;
     int32_t term_mode;
@@ -49,7 +50,7 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     size_t n = 0;
     n += 4 * (size_t)W * 2;                      // q_key, q_id
     n += 8 * (size_t)G * occ_words * 2;          // occ, end_mask
-    n += 4 * (size_t)G * (H + 1);                // Lh_s (PREDICT accumulators)
+    n += 4 * (size_t)G * (H + 1) * 2;            // Lh_s, Ch_s (PREDICT buckets: load sums, counts)
     n += 4 * (size_t)G;                          // sub_load
     n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
@@ -153,7 +154,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned char *fin_b = reinterpret_cast<unsigned char *>(end_mask + (size_t)G * OW);   // [A/8], 8-byte aligned
     unsigned char *eq_b = fin_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
     unsigned *Lh_s = reinterpret_cast<unsigned *>(eq_b + (((size_t)A8 + 15) & ~(size_t)15));   // [G][H1]
-    unsigned *sub_load = Lh_s + (size_t)G * H1;                                     // [G]
+    unsigned *Ch_s = Lh_s + (size_t)G * H1;                                         // [G][H1]
+    unsigned *sub_load = Ch_s + (size_t)G * H1;                                     // [G]
     unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
     unsigned short *pre_list = end_list + kEndList;                                 // [32]
     int *scal = reinterpret_cast<int *>(pre_list + 32);
@@ -201,7 +203,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     }
     for (int i = (2 * NT + tid) * 4; i < n_w; i += NT * 4) fetch_queue(i);
     for (int i = tid; i < G * OW; i += NT) occ[i] = g_occ[i];
-    for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
+    for (int i = tid; i < 2 * G * H1; i += NT) Lh_s[i] = 0u;      // Lh_s and Ch_s are adjacent
     for (int i = tid; i < G; i += NT) sub_load[i] = 0u;
 
     // router registers: lane owns workers lane and lane + 32
@@ -369,8 +371,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         if (timing) t_phase[1] = (unsigned)clock64();
 
         // ============ PREDICT (H > 0): c_hat maintenance + horizon projection ============
-        if (H > 0) {
-            const bool warp_uniform = (B % 32) == 0;
+        // Every running request adds (cur, 1) to the bucket (worker, floor(c_hat)); the router turns
+        // the buckets into L_g(k+h) = sum_{j >= h} T_j + h * sum_{j >= h} C_j by suffix sums.
+        if (HM > 0 && H > 0) {
 #pragma unroll 1
             for (int s_base = 0; s_base < A; s_base += NT * kUnroll) {
                 int bs[kUnroll]; float c0s[kUnroll]; int krs[kUnroll];
@@ -385,68 +388,55 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     const int s0 = s_base + u * NT + tid;
-                    if (s_base + u * NT >= A) break;               // uniform across the block
-                    const bool inr = s0 < A;
-                    const bool live = bs[u] != kEmpty;
-                    int cur = 0, nh = -1;
-                    if (live) {
-                        cur = bs[u] + k;
-                        const int t = (k - krs[u]) & 255;
-                        float c = c0s[u] - (float)t;
-                        if (t >= a.delta_T || c < a.c_floor) {
-                            const float *q = probs + (size_t)s0 * H;
-                            double surv = 1.0, cs = 0.0;
-                            if ((H & 3) == 0) {
-                                for (int h = 0; h < H; h += 4) {
+                    if (bs[u] == kEmpty) continue;
+                    const int cur = bs[u] + k;
+                    const int t = (k - krs[u]) & 255;
+                    float c = c0s[u] - (float)t;
+                    if (t >= a.delta_T || c < a.c_floor) {
+                        // refresh: p_fin = 1 - prod (1 - q_h) decides the gate; the expectation
+                        // sum_h prod_{j<h} (1 - q_j) is evaluated only when the gate is open
+                        const float *q = probs + (size_t)s0 * H;
+                        float qv[HM > 0 ? HM : 1];
+                        if ((H & 3) == 0) {
+#pragma unroll
+                            for (int h = 0; h < HM; h += 4) {
+                                if (h < H) {
                                     const float4 qq = *reinterpret_cast<const float4 *>(q + h);
-                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.x));
-                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.y));
-                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.z));
-                                    cs = __dadd_rn(cs, surv); surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qq.w));
-                                }
-                            } else {
-                                for (int h = 0; h < H; ++h) {
-                                    cs = __dadd_rn(cs, surv);
-                                    surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
+                                    qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
                                 }
                             }
-                            const double p_fin = __dsub_rn(1.0, surv);
-                            double v;
-                            if (p_fin >= (double)a.gate) {
-                                v = cs;
-                                if (v < (double)a.c_floor) v = (double)a.c_floor;
-                                if (v > (double)H) v = (double)H;
-                            } else {
-                                v = (double)H;
-                            }
-                            c = (float)v;
-                            g_chat0[s0] = c;
-                            g_kref[s0] = (uint8_t)(k & 255);
+                        } else {
+#pragma unroll
+                            for (int h = 0; h < HM; ++h) if (h < H) qv[h] = q[h];
                         }
-                        nh = (int)floorf(c);
-                        nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                    }
-                    const int g = (inr ? s0 : A - 1) / B;
-                    if (warp_uniform) {
-                        // common case: every running request of these 32 slots is counted at every
-                        // offset, so L_g(k+h) grows by (sum of loads) + h * (number of requests)
-                        const unsigned lv = __ballot_sync(kFull, live);
-                        const bool all_h = __all_sync(kFull, !live || nh == H);
-                        if (lv) {
-                            if (all_h) {
-                                const unsigned s = __reduce_add_sync(kFull, live ? (unsigned)cur : 0u);
-                                if (lane <= H) atomicAdd(&Lh_s[g * H1 + lane], s + (unsigned)(lane * __popc(lv)));
-                            } else {
-                                for (int h = 0; h <= H; ++h) {
-                                    const unsigned v = (live && h <= nh) ? (unsigned)(cur + h) : 0u;
-                                    const unsigned s = __reduce_add_sync(kFull, v);
-                                    if (lane == 0 && s) atomicAdd(&Lh_s[g * H1 + h], s);
+                        double surv = 1.0;
+#pragma unroll
+                        for (int h = 0; h < HM; ++h)
+                            if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
+                        const double p_fin = __dsub_rn(1.0, surv);
+                        double v = (double)H;
+                        if (p_fin >= (double)a.gate) {
+                            double sv = 1.0, cs = 0.0;
+#pragma unroll
+                            for (int h = 0; h < HM; ++h) {
+                                if (h < H) {
+                                    cs = __dadd_rn(cs, sv);
+                                    sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
                                 }
                             }
+                            v = cs;
+                            if (v < (double)a.c_floor) v = (double)a.c_floor;
+                            if (v > (double)H) v = (double)H;
                         }
-                    } else if (live) {
-                        for (int h = 0; h <= nh; ++h) atomicAdd(&Lh_s[g * H1 + h], (unsigned)(cur + h));
+                        c = (float)v;
+                        g_chat0[s0] = c;
+                        g_kref[s0] = (uint8_t)(k & 255);
                     }
+                    int nh = (int)floorf(c);
+                    nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                    const int g = (int)__umulhi((unsigned)s0, a.magic_B);        // s0 / B
+                    atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
+                    atomicAdd(&Ch_s[g * H1 + nh], 1u);
                 }
             }
         }
@@ -460,8 +450,12 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 for (int w = 0; w < GW; ++w) {
                     const int g = lane + 32 * w;
 #pragma unroll
-                    for (int h = 0; h <= HM; ++h)
-                        L[w][h] = (g < G && h <= H) ? (int)Lh_s[g * H1 + h] : 0;
+                    int accT = 0, accC = 0;
+#pragma unroll
+                    for (int h = HM; h >= 0; --h) {
+                        if (g < G && h <= H) { accT += (int)Lh_s[g * H1 + h]; accC += (int)Ch_s[g * H1 + h]; }
+                        L[w][h] = (g < G && h <= H) ? accT + h * accC : 0;
+                    }
                 }
             }
 #pragma unroll
@@ -863,7 +857,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             }
         }
         if (it + 1 < a.n_steps) {
-            for (int i = tid; i < G * H1; i += NT) Lh_s[i] = 0u;
+            for (int i = tid; i < 2 * G * H1; i += NT) Lh_s[i] = 0u;
             inst_sync();
         }
     }
