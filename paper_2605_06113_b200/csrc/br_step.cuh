@@ -449,7 +449,6 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 #pragma unroll
                 for (int w = 0; w < GW; ++w) {
                     const int g = lane + 32 * w;
-#pragma unroll
                     int accT = 0, accC = 0;
 #pragma unroll
                     for (int h = HM; h >= 0; --h) {

@@ -1,0 +1,48 @@
+"""br_fscore (the F-score matrix and the pool-bypass arg-max) against the checker's Eq. 1 / Eq. 2."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_06113_b200 import workload as wlm
+from paper_2605_06113_b200.binding import Router
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,H", [("c3", 0), ("c4", 8), ("c2", 4)])
+def test_fscore_matrix_and_best_worker(name, H):
+    cfg = wlm.get_config(name)
+    wl = wlm.make_workload(cfg, n_instances=2)
+    r = Router(wl, device="cuda:0")
+    rng = np.random.default_rng(3 + H)
+    N, G, n_req = 3, cfg.G, 2052                      # two full tiles and a ragged tail
+    s = rng.integers(1, 60000, (N, n_req)).astype(np.int32)
+    Lh = rng.integers(100000, 400000, (N, G, H + 1)).astype(np.int64)
+    cap = rng.integers(0, 3, (N, G)).astype(np.int32)
+    cap[2] = 0                                        # no worker has room: best_g = -1
+    st, Lt, ct = (torch.from_numpy(x).cuda() for x in (s, Lh, cap))
+    F = torch.zeros((N, n_req, G), dtype=torch.float64, device="cuda")
+    best = torch.full((N, n_req), -7, dtype=torch.int32, device="cuda")
+    r.fscore(st, Lt, F, cap=ct, best_g=best)
+    torch.cuda.synchronize()
+    Fh, bh = F.cpu().numpy(), best.cpu().numpy()
+    M = Lh.max(axis=1)                                # envelope per offset
+    for n in range(N):
+        for i in list(range(0, 40)) + list(range(n_req - 40, n_req)) + [int(x) for x in rng.integers(0, n_req, 60)]:
+            ref = np.empty(G)
+            for g in range(G):
+                m = M[n] - Lh[n, g]
+                if cfg.score_mode == 0:
+                    ref[g] = oracle.f_br0(G, int(s[n, i]), int(m[0]))
+                else:
+                    ref[g] = oracle.f_brh(H, cfg.alpha, cfg.beta, cfg.gamma, int(s[n, i]), m)
+            err = np.abs(Fh[n, i] - ref) / np.maximum(1.0, np.abs(ref))
+            assert err.max() <= 1e-6                  # stated tolerance
+            assert np.array_equal(Fh[n, i], ref)      # same arithmetic, same order: equality
+            ok = np.nonzero(cap[n] > 0)[0]
+            want = -1 if len(ok) == 0 else int(ok[np.argmax(ref[ok])])
+            assert bh[n, i] == want
+    r.close()
