@@ -44,6 +44,30 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def kernel_source_hash() -> str:
+    """Hash of the CUDA sources; the DRAM-traffic figures under profiles/ are valid only for
+    the kernel they were captured on."""
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2605_06113_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
+    profiles/traffic.json, or None if the kernel sources changed since that capture."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        rec = json.load(open(p))
+        if rec.get("kernel_source_hash") == kernel_source_hash():
+            return rec["bytes_per_launch"].get(workload)
+    except Exception:
+        pass
+    return None
+
+
 def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
     """Bytes one instance-step has to move once: running-request state in, queue in,
     assignments out, per-worker state in and out, slot edits."""
@@ -314,12 +338,13 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
 
     # ---------------- headline: c3 batched ----------------
-    cfg = wlm.get_config("c3")
+    wname = args.workload
+    cfg = wlm.get_config(wname)
     N = cfg.N
     per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
-    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
+    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state)))) if wname == "c3" else 2
     first, _ = shard_of(rank, world, N, n_sets)
-    sets = RotatingSets("c3", N, n_sets, device, seed_offset=first, threads=args.threads)
+    sets = RotatingSets(wname, N, n_sets, device, seed_offset=first, threads=args.threads, probs_ring=4)
     sampler = ClockSampler(local)
     sampler.start()
     ms = time_launches(torch, sets.step, args.warmup, args.steps, dist)
@@ -328,19 +353,22 @@ def run_ours(args):
     bad = int((sets.out["status"] & ~1).ne(0).sum().item())
     value = world * N * args.steps / (ms * 1e-3)
     # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
-    edits = float(2.0 * cnt[1] + 10.0)
-    abytes = algorithmic_bytes(cfg, edits, 0.0) * N
+    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
+    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N
     achieved = abytes / (ms * 1e-3 / args.steps) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "peak_kind": peak_kind, "traffic": None,
-                "algorithmic_bytes_per_launch": abytes, "kernel": "br_step_kernel<false,0>"}
+                "peak_kind": peak_kind, "traffic": recorded_traffic(wname),
+                "algorithmic_bytes_per_launch": abytes,
+                "kernel": "br_step_kernel<false,0,1>" if wname == "c3" else "br_step_kernel<true,8,2>"}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
+        "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100..",
+        "config": {"workload": ("c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.." if wname == "c3"
+                                else "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000.."),
                    "instances_per_launch": N, "rotating_sets": n_sets,
                    "l2": f"{n_sets} instance sets stepped in rotation: data touched between two visits "
                          f"of a set exceeds the 126 MB L2", "threads_per_instance": sets.router.params.threads},
@@ -348,7 +376,7 @@ def run_ours(args):
         "bad_status_instances": bad,
     }
 
-    if rank == 0 and world == 1 and not args.quick:
+    if rank == 0 and world == 1 and not args.quick and wname == "c3":
         # ---------------- end to end through the host-buffer entry point ----------------
         line["e2e"] = e2e_host(torch, device, args)
         # ---------------- extras: c4 batched BR-H, latency path ----------------
@@ -357,9 +385,9 @@ def run_ours(args):
         except Exception as ex:  # keep the headline line even if an extra fails
             line["extra"] = {"error": repr(ex)}
         # ---------------- CPU baseline: the checker on host cores ----------------
-        rate, done, dt = oracle_rate("c3", 12.0, 64, 500)
+        rate, done, dt = oracle_rate("c3", 12.0, 512, 500)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{done} instance-steps of c3 (first 64 instances, steps 0..{done // 64 - 1}), "
+                                "sample": f"{done} instance-steps of c3 (first 512 instances, steps 0..{done // 512 - 1}), "
                                           f"{dt:.1f} s, single thread"}
     elif rank == 0:
         line["e2e"] = None
@@ -404,7 +432,8 @@ def extras(torch, device, args, peak):
     ach = abytes / (ms * 1e-3 / 200) / 1e9
     ex["c4_batched"] = {"value": cfg.N * 200 / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / 200,
                         "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                                     "frac": ach / peak, "algorithmic_bytes_per_launch": abytes}}
+                                     "frac": ach / peak, "traffic": recorded_traffic("c4"),
+                                     "algorithmic_bytes_per_launch": abytes}}
     del sets
     torch.cuda.empty_cache()
     # c3 with 16 steps per launch (persistent multi-step form of the same kernel)
@@ -421,6 +450,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="headline measurement only")
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4"],
+                    help="batched configuration timed as the headline (c4 is used for profiling the BR-H kernel)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
