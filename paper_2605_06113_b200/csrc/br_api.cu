@@ -80,7 +80,8 @@ int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_work
     if (misaligned(ws->act_base, 16) || misaligned(wq->s, 16) || misaligned(wq->id, 16) ||
         misaligned(assign_out, 16) || misaligned(ws->load, 8) || misaligned(ws->occ, 8) ||
         misaligned(out->load, 8) || misaligned(out->trace, 8) || misaligned(ws->seed, 8) ||
-        (term_probs && misaligned(term_probs, 16)) || (out->fscore && misaligned(out->fscore, 8)))
+        (term_probs && misaligned(term_probs, 16)) || (out->fscore && misaligned(out->fscore, 8)) ||
+        (ctx->H > 0 && (misaligned(ws->act_chat0, 16) || misaligned(ws->act_kref, 4))))
         return BR_EINVAL;
     return BR_OK;
 }

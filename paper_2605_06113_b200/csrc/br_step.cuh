@@ -122,7 +122,7 @@ __device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
     return (x - 0x00010001u * n) & ~x & 0x80008000u;
 }
 
-constexpr int kUnroll = 4;      // loads in flight per thread in the BR-H streaming phase
+constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
 template <bool FP, int HM, int GW>
@@ -374,24 +374,32 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // Every running request adds (cur, 1) to the bucket (worker, floor(c_hat)); the router turns
         // the buckets into L_g(k+h) = sum_{j >= h} T_j + h * sum_{j >= h} C_j by suffix sums.
         if (HM > 0 && H > 0) {
+            const int A4 = A >> 2;
 #pragma unroll 1
-            for (int s_base = 0; s_base < A; s_base += NT * kUnroll) {
-                int bs[kUnroll]; float c0s[kUnroll]; int krs[kUnroll];
+            for (int q_base = 0; q_base < A4; q_base += NT * kUnroll) {
+                // four consecutive slots per thread and 16-byte loads, kUnroll quads in flight
+                int4 bq[kUnroll]; float4 cq[kUnroll]; unsigned kq[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    const int s0 = s_base + u * NT + tid;
-                    const bool inr = s0 < A;
-                    bs[u] = inr ? g_base[s0] : kEmpty;
-                    c0s[u] = inr ? g_chat0[s0] : 0.0f;
-                    krs[u] = inr ? (int)g_kref[s0] : 0;
+                    const int q4 = q_base + u * NT + tid;
+                    const bool inr = q4 < A4;
+                    bq[u] = inr ? *reinterpret_cast<const int4 *>(g_base + 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
+                    cq[u] = inr ? *reinterpret_cast<const float4 *>(g_chat0 + 4 * q4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    kq[u] = inr ? *reinterpret_cast<const unsigned *>(g_kref + 4 * q4) : 0u;
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    const int s0 = s_base + u * NT + tid;
-                    if (bs[u] == kEmpty) continue;
-                    const int cur = bs[u] + k;
-                    const int t = (k - krs[u]) & 255;
-                    float c = c0s[u] - (float)t;
+                  const int q4 = q_base + u * NT + tid;
+                  const int bs4[4] = {bq[u].x, bq[u].y, bq[u].z, bq[u].w};
+                  const float c04[4] = {cq[u].x, cq[u].y, cq[u].z, cq[u].w};
+                  const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);      // slot / B
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const int s0 = 4 * q4 + j;
+                    if (bs4[j] == kEmpty) continue;
+                    const int cur = bs4[j] + k;
+                    const int t = (k - (int)((kq[u] >> (8 * j)) & 0xFFu)) & 255;
+                    float c = c04[j] - (float)t;
                     if (t >= a.delta_T || c < a.c_floor) {
                         // refresh: p_fin = 1 - prod (1 - q_h) decides the gate; the expectation
                         // sum_h prod_{j<h} (1 - q_j) is evaluated only when the gate is open
@@ -434,9 +442,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     }
                     int nh = (int)floorf(c);
                     nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                    const int g = (int)__umulhi((unsigned)s0, a.magic_B);        // s0 / B
                     atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
                     atomicAdd(&Ch_s[g * H1 + nh], 1u);
+                  }
                 }
             }
         }
