@@ -63,6 +63,7 @@ template <bool FP, int HM>
 struct Scorer {
     int mi;                 // Eq. 1 margin
     double md[HM + 1];      // Eq. 2 margins
+    int mmin;               // min_h m_{g,h}: at or below it the Eq. 2 penalty is exactly zero
 
     __device__ __forceinline__ long long key(const StepArgs &a, int delta) const
     {
@@ -417,11 +418,21 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 #pragma unroll
                             for (int h = 0; h < HM; ++h) if (h < H) qv[h] = q[h];
                         }
-                        double surv = 1.0;
+                        // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
+                        // clearly below the gate the fp64 product cannot reach it and is not evaluated
+                        float qsum = 0.0f, qmin = 0.0f;
 #pragma unroll
-                        for (int h = 0; h < HM; ++h)
-                            if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
-                        const double p_fin = __dsub_rn(1.0, surv);
+                        for (int h = 0; h < HM; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
+                        double p_fin = 0.0;
+                        if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
+                            double surv = 1.0;
+#pragma unroll
+                            for (int h = 0; h < HM; ++h)
+                                if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
+                            p_fin = __dsub_rn(1.0, surv);
+                        } else if (a.gate <= 0.0f) {
+                            p_fin = 1.0;
+                        }
                         double v = (double)H;
                         if (p_fin >= (double)a.gate) {
                             double sv = 1.0, cs = 0.0;
@@ -484,13 +495,17 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[0] - L[w][0];
                     sc.mi = __shfl_sync(kFull, mine, src);
                 } else {
+                    int mmin = 0x7FFFFFFF;
 #pragma unroll
                     for (int h = 0; h <= HM; ++h) {
                         int mine = Mh[h] - L[0][h];
 #pragma unroll
                         for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[h] - L[w][h];
-                        sc.md[h] = (double)__shfl_sync(kFull, mine, src);
+                        const int mh = __shfl_sync(kFull, mine, src);
+                        sc.md[h] = (double)mh;
+                        if (h <= H) mmin = min(mmin, mh);
                     }
+                    sc.mmin = mmin;
                 }
             };
 
@@ -532,14 +547,26 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int res = __shfl_sync(kFull, bkey, src);
                     return res > 0 ? res : 0;
                 } else {
-                    long long bk = kNoKey; int bkey = 0;
-#pragma unroll 1
+                    // Horizon-safe requests (s <= min_h m_{g,h}) score alpha D s exactly, which grows
+                    // with s: of those only the largest key per lane is scored; the others in full.
+                    long long bk = kNoKey; int bkey = 0, best_safe = 0;
+#pragma unroll 2
                     for (int t = 0; t < n_tiles; ++t) {
                         const int idx = (t << 5) + lane;
                         const int qk = idx < n_w ? q_key[idx] : 0;
                         if (qk > 0) {
-                            const long long f = sc.key(a, qk >> WL);
-                            if (f > bk) { bk = f; bkey = qk; }
+                            if ((qk >> WL) <= sc.mmin) {
+                                best_safe = max(best_safe, qk);
+                            } else {
+                                const long long f = sc.key(a, qk >> WL);
+                                if (f > bk) { bk = f; bkey = qk; }
+                            }
+                        }
+                    }
+                    if (best_safe > 0) {
+                        const long long f = sc.key(a, best_safe >> WL);
+                        if (f > bk || (f == bk && ((unsigned)best_safe & posmask) > ((unsigned)bkey & posmask))) {
+                            bk = f; bkey = best_safe;
                         }
                     }
                     long long wk;
