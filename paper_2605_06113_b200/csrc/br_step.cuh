@@ -54,6 +54,7 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     n += 4 * (size_t)G;                          // sub_load
     n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
+    if (H > 0) n += 2 * (size_t)G * B;           // refresh_list
     return (n + 15) & ~(size_t)15;
 }
 
@@ -160,9 +161,11 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
     unsigned short *pre_list = end_list + kEndList;                                 // [32]
     int *scal = reinterpret_cast<int *>(pre_list + 32);
+    unsigned short *refresh_list = reinterpret_cast<unsigned short *>(scal + 16);   // [A] (H > 0 only)
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
-    //       [6] requests that ended this step and were not prefetched, [7] prefetched ones
+    //       [6] requests that ended this step and were not prefetched, [7] prefetched ones,
+    //       [8] requests whose c_hat is refreshed at this step
 
     // ---- per-instance global rows ----
     long long *g_load = reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G;
@@ -374,11 +377,12 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // ============ PREDICT (H > 0): c_hat maintenance + horizon projection ============
         // Every running request adds (cur, 1) to the bucket (worker, floor(c_hat)); the router turns
         // the buckets into L_g(k+h) = sum_{j >= h} T_j + h * sum_{j >= h} C_j by suffix sums.
+        // Pass A streams the per-request state and settles the requests that only age; the ones due
+        // for a refresh are listed, and pass B reads their classifier rows with independent loads.
         if (HM > 0 && H > 0) {
             const int A4 = A >> 2;
 #pragma unroll 1
             for (int q_base = 0; q_base < A4; q_base += NT * kUnroll) {
-                // four consecutive slots per thread and 16-byte loads, kUnroll quads in flight
                 int4 bq[kUnroll]; float4 cq[kUnroll]; unsigned kq[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
@@ -390,73 +394,89 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                  const int q4 = q_base + u * NT + tid;
-                  const int bs4[4] = {bq[u].x, bq[u].y, bq[u].z, bq[u].w};
-                  const float c04[4] = {cq[u].x, cq[u].y, cq[u].z, cq[u].w};
-                  const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);      // slot / B
+                    const int q4 = q_base + u * NT + tid;
+                    const int bs4[4] = {bq[u].x, bq[u].y, bq[u].z, bq[u].w};
+                    const float c04[4] = {cq[u].x, cq[u].y, cq[u].z, cq[u].w};
+                    const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);      // slot / B
 #pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    const int s0 = 4 * q4 + j;
-                    if (bs4[j] == kEmpty) continue;
-                    const int cur = bs4[j] + k;
-                    const int t = (k - (int)((kq[u] >> (8 * j)) & 0xFFu)) & 255;
-                    float c = c04[j] - (float)t;
-                    if (t >= a.delta_T || c < a.c_floor) {
-                        // refresh: p_fin = 1 - prod (1 - q_h) decides the gate; the expectation
-                        // sum_h prod_{j<h} (1 - q_j) is evaluated only when the gate is open
-                        const float *q = probs + (size_t)s0 * H;
-                        float qv[HM > 0 ? HM : 1];
-                        if ((H & 3) == 0) {
-#pragma unroll
-                            for (int h = 0; h < HM; h += 4) {
-                                if (h < H) {
-                                    const float4 qq = *reinterpret_cast<const float4 *>(q + h);
-                                    qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
-                                }
-                            }
-                        } else {
-#pragma unroll
-                            for (int h = 0; h < HM; ++h) if (h < H) qv[h] = q[h];
+                    for (int j = 0; j < 4; ++j) {
+                        const bool live = bs4[j] != kEmpty;
+                        const int t = (k - (int)((kq[u] >> (8 * j)) & 0xFFu)) & 255;
+                        const float c = c04[j] - (float)t;
+                        const bool due = live && (t >= a.delta_T || c < a.c_floor);
+                        const unsigned dm = __ballot_sync(kFull, due);          // one list append per warp
+                        if (dm) {
+                            const int lead = __ffs(dm) - 1;
+                            int at = 0;
+                            if (lane == lead) at = atomicAdd(&scal[8], __popc(dm));
+                            at = __shfl_sync(kFull, at, lead);
+                            if (due) refresh_list[at + __popc(dm & ((1u << lane) - 1u))] = (unsigned short)(4 * q4 + j);
                         }
-                        // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
-                        // clearly below the gate the fp64 product cannot reach it and is not evaluated
-                        float qsum = 0.0f, qmin = 0.0f;
-#pragma unroll
-                        for (int h = 0; h < HM; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
-                        double p_fin = 0.0;
-                        if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
-                            double surv = 1.0;
-#pragma unroll
-                            for (int h = 0; h < HM; ++h)
-                                if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
-                            p_fin = __dsub_rn(1.0, surv);
-                        } else if (a.gate <= 0.0f) {
-                            p_fin = 1.0;
+                        if (live && !due) {
+                            int nh = (int)floorf(c);
+                            nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                            atomicAdd(&Lh_s[g * H1 + nh], (unsigned)(bs4[j] + k));
+                            atomicAdd(&Ch_s[g * H1 + nh], 1u);
                         }
-                        double v = (double)H;
-                        if (p_fin >= (double)a.gate) {
-                            double sv = 1.0, cs = 0.0;
-#pragma unroll
-                            for (int h = 0; h < HM; ++h) {
-                                if (h < H) {
-                                    cs = __dadd_rn(cs, sv);
-                                    sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
-                                }
-                            }
-                            v = cs;
-                            if (v < (double)a.c_floor) v = (double)a.c_floor;
-                            if (v > (double)H) v = (double)H;
-                        }
-                        c = (float)v;
-                        g_chat0[s0] = c;
-                        g_kref[s0] = (uint8_t)(k & 255);
                     }
-                    int nh = (int)floorf(c);
-                    nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                    atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
-                    atomicAdd(&Ch_s[g * H1 + nh], 1u);
-                  }
                 }
+            }
+            inst_sync();
+            const int n_ref = scal[8];
+#pragma unroll 2
+            for (int e = tid; e < n_ref; e += NT) {
+                const int s0 = refresh_list[e];
+                const float *q = probs + (size_t)s0 * H;
+                float qv[HM > 0 ? HM : 1];
+                if ((H & 3) == 0) {
+#pragma unroll
+                    for (int h = 0; h < HM; h += 4) {
+                        if (h < H) {
+                            const float4 qq = *reinterpret_cast<const float4 *>(q + h);
+                            qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < HM; ++h) if (h < H) qv[h] = q[h];
+                }
+                const int cur = g_base[s0] + k;
+                // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
+                // clearly below the gate the fp64 product cannot reach it and is not evaluated
+                float qsum = 0.0f, qmin = 0.0f;
+#pragma unroll
+                for (int h = 0; h < HM; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
+                double p_fin = 0.0;
+                if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
+                    double surv = 1.0;
+#pragma unroll
+                    for (int h = 0; h < HM; ++h)
+                        if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
+                    p_fin = __dsub_rn(1.0, surv);
+                }
+                double v = (double)H;
+                if (p_fin >= (double)a.gate) {
+                    // gate open: E[min(r, H)] = sum_h prod_{j<h} (1 - q_j), clipped to [floor, H]
+                    double sv = 1.0, cs = 0.0;
+#pragma unroll
+                    for (int h = 0; h < HM; ++h) {
+                        if (h < H) {
+                            cs = __dadd_rn(cs, sv);
+                            sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
+                        }
+                    }
+                    v = cs;
+                    if (v < (double)a.c_floor) v = (double)a.c_floor;
+                    if (v > (double)H) v = (double)H;
+                }
+                const float c = (float)v;
+                g_chat0[s0] = c;
+                g_kref[s0] = (uint8_t)(k & 255);
+                int nh = (int)floorf(c);
+                nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                const int g = (int)__umulhi((unsigned)s0, a.magic_B);
+                atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
+                atomicAdd(&Ch_s[g * H1 + nh], 1u);
             }
         }
         inst_sync();                                              // B1
@@ -879,7 +899,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     c[0] = (uint32_t)n_drop; c[1] = (uint32_t)scal[1]; c[2] = (uint32_t)scal[2]; c[3] = (uint32_t)scal[3];
                 }
                 if (a.out.status) a.out.status[orow] = scal[4] | scal[5];
-                scal[6] = 0; scal[7] = 0;
+                scal[6] = 0; scal[7] = 0; scal[8] = 0;
                 if (timing) {
                     t_phase[6] = (unsigned)clock64();
                     uint32_t *pc = a.out.phase_cycles + orow * 8;
