@@ -547,6 +547,12 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             int admitted = 0, s1_iters = 0, s2_pops = 0, status = 0;
             const int n_tiles = (n_w + 31) >> 5;
 
+            // Stage-2 window state: each lane's five largest waiting keys, sorted, built by the first
+            // pop of the step and kept up to date as requests are admitted
+            int wt0 = 0, wt1 = 0, wt2 = 0, wt3 = 0, wt4 = 0;
+            bool w_built = false, w_trunc = false;
+            constexpr bool w_keep = FP;       // Eq. 1 kernels rescan at every pop: less code, and their scans are cheap
+
             // argmax_i F_g({i}) over all waiting requests, earliest arrival on ties.
             // Returns the packed key of the winner (0 if none).
             auto best_single = [&]() -> int {
@@ -640,6 +646,13 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         Mh[h] = max(Mh[h], __shfl_sync(kFull, mine, src));
                     }
                 }
+                if (w_keep && w_built && lane == (pos & 31)) {
+                    if (wt0 == qk) { wt0 = wt1; wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
+                    else if (wt1 == qk) { wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
+                    else if (wt2 == qk) { wt2 = wt3; wt3 = wt4; wt4 = 0; }
+                    else if (wt3 == qk) { wt3 = wt4; wt4 = 0; }
+                    else if (wt4 == qk) { wt4 = 0; }
+                }
                 __syncwarp();
                 S_tot -= 1; n_left -= 1; admitted += 1;
             };
@@ -688,31 +701,48 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int g = (int)mg;
                     load_margins(g);
 
-                    // window: the R_max largest waiting requests, earliest first on ties.
-                    // One pass keeps each lane's four largest keys sorted; the heads are merged.
-                    int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0;
-#pragma unroll 4
-                    for (int t = 0; t < n_tiles; ++t) {
-                        const int idx = (t << 5) + lane;
-                        int x = idx < n_w ? q_key[idx] : 0;
-                        int y;
-                        y = max(t0, x); x = min(t0, x); t0 = y;
-                        y = max(t1, x); x = min(t1, x); t1 = y;
-                        y = max(t2, x); x = min(t2, x); t2 = y;
-                        y = max(t3, x); x = min(t3, x); t3 = y;
-                        t4 = max(t4, x);
-                    }
+                    // window: the R_max largest waiting requests, earliest first on ties: the heads of
+                    // the lanes' sorted lists are merged.  A list that runs dry although its lane holds
+                    // more keys (possible only after several admissions from one lane) forces a rebuild.
                     int win[BR_MAX_RMAX];
                     int nwin = 0;
-#pragma unroll
-                    for (int r = 0; r < BR_MAX_RMAX; ++r) {
-                        win[r] = 0;
-                        if (r < a.R_max && r < n_left) {
-                            const int m = __reduce_max_sync(kFull, t0);
-                            win[r] = m;
-                            if (m > 0) nwin = r + 1;
-                            if (t0 == m) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = 0; }
+#pragma unroll 1
+                    for (int attempt = 0; attempt < 2; ++attempt) {
+                        if (!w_built) {
+                            int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0, cnt = 0;
+#pragma unroll 4
+                            for (int t = 0; t < n_tiles; ++t) {
+                                const int idx = (t << 5) + lane;
+                                int x = idx < n_w ? q_key[idx] : 0;
+                                cnt += x > 0;
+                                int y;
+                                y = max(t0, x); x = min(t0, x); t0 = y;
+                                y = max(t1, x); x = min(t1, x); t1 = y;
+                                y = max(t2, x); x = min(t2, x); t2 = y;
+                                y = max(t3, x); x = min(t3, x); t3 = y;
+                                t4 = max(t4, x);
+                            }
+                            wt0 = t0; wt1 = t1; wt2 = t2; wt3 = t3; wt4 = t4;
+                            w_trunc = cnt > 5;
+                            w_built = true;
                         }
+                        int h0 = wt0, h1 = wt1, h2 = wt2, h3 = wt3, h4 = wt4;
+                        bool dry = false;
+                        nwin = 0;
+#pragma unroll
+                        for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                            win[r] = 0;
+                            if (r < a.R_max && r < n_left) {
+                                dry = dry || (h0 == 0 && w_trunc);
+                                const int m = __reduce_max_sync(kFull, h0);
+                                win[r] = m;
+                                if (m > 0) nwin = r + 1;
+                                if (h0 == m) { h0 = h1; h1 = h2; h2 = h3; h3 = h4; h4 = 0; }
+                            }
+                        }
+                        if (!w_keep) { w_built = false; break; }
+                        if (!__any_sync(kFull, dry)) break;
+                        w_built = false;
                     }
                     // subsets of the window: lane = mask, lowest mask on ties
                     const int lim = min(mc, a.R_max);
