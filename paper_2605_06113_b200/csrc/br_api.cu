@@ -49,18 +49,18 @@ inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintp
 typedef void (*step_kernel_t)(const StepArgs);
 
 template <int GW>
-step_kernel_t pick_kernel_gw(bool fp, int H)
+step_kernel_t pick_kernel_gw(bool fp, int H, bool lean)
 {
-    if (!fp) return br::br_step_kernel<false, 0, GW>;
-    if (H == 0) return br::br_step_kernel<true, 0, GW>;
-    if (H <= 4) return br::br_step_kernel<true, 4, GW>;
-    if (H <= 8) return br::br_step_kernel<true, 8, GW>;
-    return br::br_step_kernel<true, 16, GW>;
+    if (!fp) return lean ? br::br_step_kernel<false, 0, GW, true> : br::br_step_kernel<false, 0, GW, false>;
+    if (H == 0) return br::br_step_kernel<true, 0, GW, false>;
+    if (H <= 4) return br::br_step_kernel<true, 4, GW, false>;
+    if (H <= 8) return br::br_step_kernel<true, 8, GW, false>;
+    return br::br_step_kernel<true, 16, GW, false>;
 }
 
-step_kernel_t pick_kernel(bool fp, int H, int G)
+step_kernel_t pick_kernel(bool fp, int H, int G, bool lean)
 {
-    return G <= 32 ? pick_kernel_gw<1>(fp, H) : pick_kernel_gw<2>(fp, H);
+    return G <= 32 ? pick_kernel_gw<1>(fp, H, lean) : pick_kernel_gw<2>(fp, H, lean);
 }
 
 int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_worker_state *ws,
@@ -99,9 +99,10 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.term_probs = term_probs;
     a.assign_out = assign_out;
     a.out = *out;
-    step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G);
     // few instances: the launch is latency-bound, so spread each instance over more warps
     const int tpi = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
+    const bool lean = tpi == 32 && ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles;
+    step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
     // single-warp instances are packed several to a block
     int per_block = (tpi == 32) ? ctx->inst_per_block : 1;
     if (per_block > b->n_instances) per_block = b->n_instances;

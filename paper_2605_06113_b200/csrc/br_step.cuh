@@ -127,7 +127,9 @@ __device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
 constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
-template <bool FP, int HM, int GW>
+// LEAN: a single-warp instance with constant-hazard terminations and no optional outputs (score
+// matrix, cycle counters); the other paths are compiled out, which shortens the code every warp walks.
+template <bool FP, int HM, int GW, bool LEAN>
 __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const StepArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_all[];
@@ -139,7 +141,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     if (blockIdx.x * per_block + in_block >= a.N) return;            // whole instance groups only
     unsigned char *smem_raw = smem_all + (size_t)in_block * a.smem_per_inst;
     auto inst_sync = [&]() { if (NT == 32) __syncwarp(); else __syncthreads(); };
-    const int nwarps = NT >> 5;
+    const int nwarps = LEAN ? 1 : (NT >> 5);
+    const int term_mode = LEAN ? 1 : a.term_mode;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
     const int A8 = A >> 3;
     const int WL = a.wl;
@@ -272,7 +275,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             const int g = idx / OW, x = idx - g * OW;
             const unsigned long long occw = occ[idx];
             unsigned long long finw = 0ull, eqw = 0ull;
-            if (a.term_mode != 0 && occw) {
+            if (term_mode != 0 && occw) {
                 const int b0 = g * (B >> 3) + 8 * x;
                 const int nb = min(8, (B >> 3) - 8 * x);
                 if (nb == 8 && (b0 & 7) == 0) {
@@ -319,7 +322,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         const size_t orow = (size_t)it * a.N + inst;
         const float *probs = a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr;
         unsigned t_phase[7];
-        const bool timing = a.out.phase_cycles != nullptr && tid == 0;
+        const bool timing = !LEAN && a.out.phase_cycles != nullptr && tid == 0;
         if (timing) t_phase[0] = (unsigned)clock64();
 
         // ================= ARRIVE =================
@@ -335,7 +338,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // A single-warp instance also resolves, right away, which of the requests already
         // running end at this step, and requests their loads: the values are used only after
         // routing, so that memory latency is off the step's critical path.
-        const bool have_pre = (nwarps == 1 && a.term_mode == 1);
+        const bool have_pre = (nwarps == 1 && term_mode == 1);
         int pend = 0, n_pre = 0;
         if (have_pre) {
             draw_terms(tid, NT);
@@ -530,7 +533,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             };
 
             // optional F-score matrix before the first admission
-            if (a.out.fscore) {
+            if (!LEAN && a.out.fscore) {
                 double *F = a.out.fscore + orow * (size_t)W * G;
                 for (int g = 0; g < G; ++g) {
                     load_margins(g);
@@ -795,7 +798,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     scal[4] = status | (n_drop ? BR_ST_QUEUE_OVERFLOW : 0);
                 }
             }
-        } else if (a.term_mode == 1) {
+        } else if (term_mode == 1) {
             // warps 1.. draw this step's termination words while warp 0 routes
             draw_terms(tid - 32, NT - 32);
         }
@@ -858,7 +861,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // ================= ADVANCE =================
         // Only the occupancy masks, the termination draws and the few ending slots are touched.
         if (!have_pre) {
-            if (a.term_mode == 2) {
+            if (term_mode == 2) {
                 // Bernoulli(term_probs[slot][0]) per running request: 24-bit uniform below the probability
                 const float sc24 = 5.9604644775390625e-8f;
 #pragma unroll 1
