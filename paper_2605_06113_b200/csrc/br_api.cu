@@ -108,6 +108,7 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     if (per_block > b->n_instances) per_block = b->n_instances;
     while (per_block > 1 && ctx->smem * per_block > 48 * 1024) --per_block;
     a.tpi = tpi;
+    a.block_sync = (per_block > 1 && b->n_instances % per_block == 0) ? 1 : 0;
     a.smem_per_inst = (int32_t)ctx->smem;
     const int blocks = (b->n_instances + per_block - 1) / per_block;
     kern<<<blocks, tpi * per_block, ctx->smem * per_block, stream>>>(a);

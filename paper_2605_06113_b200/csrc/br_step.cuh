@@ -37,6 +37,7 @@ struct StepArgs {
     double d[BR_MAX_H + 1];
     int32_t N, first_instance, n_steps;
     int32_t tpi, smem_per_inst;  // threads and shared-memory bytes per instance
+    int32_t block_sync;          // 1: every barrier is a block barrier (needs full blocks)
     br_worker_state ws;
     br_waiting_queue wq;
     const float *term_probs;
@@ -140,7 +141,10 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     const int in_block = threadIdx.x / NT, per_block = blockDim.x / NT;
     if (blockIdx.x * per_block + in_block >= a.N) return;            // whole instance groups only
     unsigned char *smem_raw = smem_all + (size_t)in_block * a.smem_per_inst;
-    auto inst_sync = [&]() { if (NT == 32) __syncwarp(); else __syncthreads(); };
+    // Instance-wide barrier.  Single-warp instances that share a block may also be aligned with a
+    // block barrier (a.block_sync): the warps then walk the same code at about the same time, which
+    // pays off in instruction fetch although no data crosses between them.
+    auto inst_sync = [&]() { if (NT == 32 && !a.block_sync) __syncwarp(); else __syncthreads(); };
     const int nwarps = LEAN ? 1 : (NT >> 5);
     const int term_mode = LEAN ? 1 : a.term_mode;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
