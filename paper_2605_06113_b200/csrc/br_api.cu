@@ -48,17 +48,18 @@ inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintp
 
 typedef void (*step_kernel_t)(const StepArgs);
 
+// lean: 0 general, 1 constant hazard and no optional outputs, 2 the same on a single warp
 template <int GW>
-step_kernel_t pick_kernel_gw(bool fp, int H, bool lean)
+step_kernel_t pick_kernel_gw(bool fp, int H, int lean)
 {
-    if (!fp) return lean ? br::br_step_kernel<false, 0, GW, true> : br::br_step_kernel<false, 0, GW, false>;
-    if (H == 0) return br::br_step_kernel<true, 0, GW, false>;
-    if (H <= 4) return br::br_step_kernel<true, 4, GW, false>;
-    if (H <= 8) return br::br_step_kernel<true, 8, GW, false>;
-    return br::br_step_kernel<true, 16, GW, false>;
+    if (!fp) return lean == 2 ? br::br_step_kernel<false, 0, GW, 2> : br::br_step_kernel<false, 0, GW, 0>;
+    if (H == 0) return br::br_step_kernel<true, 0, GW, 0>;
+    if (H <= 4) return lean ? br::br_step_kernel<true, 4, GW, 1> : br::br_step_kernel<true, 4, GW, 0>;
+    if (H <= 8) return lean ? br::br_step_kernel<true, 8, GW, 1> : br::br_step_kernel<true, 8, GW, 0>;
+    return lean ? br::br_step_kernel<true, 16, GW, 1> : br::br_step_kernel<true, 16, GW, 0>;
 }
 
-step_kernel_t pick_kernel(bool fp, int H, int G, bool lean)
+step_kernel_t pick_kernel(bool fp, int H, int G, int lean)
 {
     return G <= 32 ? pick_kernel_gw<1>(fp, H, lean) : pick_kernel_gw<2>(fp, H, lean);
 }
@@ -101,7 +102,7 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.out = *out;
     // few instances: the launch is latency-bound, so spread each instance over more warps
     const int tpi = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
-    const bool lean = tpi == 32 && ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles;
+    const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles) ? (tpi == 32 ? 2 : 1) : 0;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
     // single-warp instances are packed several to a block
     int per_block = (tpi == 32) ? ctx->inst_per_block : 1;

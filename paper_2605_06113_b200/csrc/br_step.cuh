@@ -128,9 +128,10 @@ __device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
 constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
-// LEAN: a single-warp instance with constant-hazard terminations and no optional outputs (score
-// matrix, cycle counters); the other paths are compiled out, which shortens the code every warp walks.
-template <bool FP, int HM, int GW, bool LEAN>
+// LEAN > 0: constant-hazard terminations and no optional outputs (score matrix, cycle counters);
+// LEAN == 2: in addition the instance is a single warp.  The paths not needed are compiled out,
+// which shortens the code every warp walks.
+template <bool FP, int HM, int GW, int LEAN>
 __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const StepArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_all[];
@@ -145,7 +146,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     // block barrier (a.block_sync): the warps then walk the same code at about the same time, which
     // pays off in instruction fetch although no data crosses between them.
     auto inst_sync = [&]() { if (NT == 32 && !a.block_sync) __syncwarp(); else __syncthreads(); };
-    const int nwarps = LEAN ? 1 : (NT >> 5);
+    const int nwarps = LEAN == 2 ? 1 : (NT >> 5);
     const int term_mode = LEAN ? 1 : a.term_mode;
     const int G = a.G, H = a.H, B = a.B, W = a.W, H1 = H + 1, A = G * B, OW = a.occ_words;
     const int A8 = A >> 3;
