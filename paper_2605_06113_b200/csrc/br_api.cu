@@ -105,9 +105,13 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles) ? (tpi == 32 ? 2 : 1) : 0;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
     // single-warp instances are packed several to a block
-    int per_block = (tpi == 32) ? ctx->inst_per_block : 1;
+    // instances are packed several to a block: single-warp ones always, wider ones only in full
+    // blocks (their barriers are block barriers)
+    int per_block = ctx->inst_per_block;
+    if (tpi > 32) { while (per_block > 1 && (per_block * tpi > 256 || b->n_instances % per_block != 0)) --per_block; }
     if (per_block > b->n_instances) per_block = b->n_instances;
     while (per_block > 1 && ctx->smem * per_block > 48 * 1024) --per_block;
+    if (tpi > 32 && per_block > 1 && b->n_instances % per_block != 0) per_block = 1;
     a.tpi = tpi;
     a.block_sync = (per_block > 1 && b->n_instances % per_block == 0) ? 1 : 0;
     a.smem_per_inst = (int32_t)ctx->smem;
