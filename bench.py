@@ -360,7 +360,7 @@ def run_ours(args):
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "peak_kind": peak_kind, "traffic": recorded_traffic(wname),
                 "algorithmic_bytes_per_launch": abytes,
-                "kernel": "br_step_kernel<false,0,1>" if wname == "c3" else "br_step_kernel<true,8,2>"}
+                "kernel": "br_step_kernel<false,0,1,2>" if wname == "c3" else "br_step_kernel<true,8,2,1>"}
 
     line = {
         "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
