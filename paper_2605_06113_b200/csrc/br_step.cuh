@@ -559,7 +559,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             // pop of the step and kept up to date as requests are admitted
             int wt0 = 0, wt1 = 0, wt2 = 0, wt3 = 0, wt4 = 0;
             bool w_built = false, w_trunc = false;
-            constexpr bool w_keep = FP;       // Eq. 1 kernels rescan at every pop: less code, and their scans are cheap
+            constexpr bool w_keep = FP;
+            int gw[BR_MAX_RMAX] = {0, 0, 0, 0, 0};
+            bool gw_valid = false;
 
             // argmax_i F_g({i}) over all waiting requests, earliest arrival on ties.
             // Returns the packed key of the winner (0 if none).
@@ -654,6 +656,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         Mh[h] = max(Mh[h], __shfl_sync(kFull, mine, src));
                     }
                 }
+                if (!w_keep && qk >= gw[BR_MAX_RMAX - 1]) gw_valid = false;   // one of the cached largest keys leaves
                 if (w_keep && w_built && lane == (pos & 31)) {
                     if (wt0 == qk) { wt0 = wt1; wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
                     else if (wt1 == qk) { wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
@@ -709,20 +712,18 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int g = (int)mg;
                     load_margins(g);
 
-                    // window: the R_max largest waiting requests, earliest first on ties: the heads of
-                    // the lanes' sorted lists are merged.  A list that runs dry although its lane holds
-                    // more keys (possible only after several admissions from one lane) forces a rebuild.
+                    // window: the R_max largest waiting requests, earliest first on ties
                     int win[BR_MAX_RMAX];
                     int nwin = 0;
-#pragma unroll 1
-                    for (int attempt = 0; attempt < 2; ++attempt) {
-                        if (!w_built) {
-                            int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0, cnt = 0;
+                    if (!w_keep) {
+                        // Eq. 1 kernels cache the five largest keys of the queue; the cache stays valid
+                        // until one of them is admitted (the guard mostly admits small requests)
+                        if (!gw_valid) {
+                            int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0;
 #pragma unroll 4
                             for (int t = 0; t < n_tiles; ++t) {
                                 const int idx = (t << 5) + lane;
                                 int x = idx < n_w ? q_key[idx] : 0;
-                                cnt += x > 0;
                                 int y;
                                 y = max(t0, x); x = min(t0, x); t0 = y;
                                 y = max(t1, x); x = min(t1, x); t1 = y;
@@ -730,27 +731,60 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                                 y = max(t3, x); x = min(t3, x); t3 = y;
                                 t4 = max(t4, x);
                             }
-                            wt0 = t0; wt1 = t1; wt2 = t2; wt3 = t3; wt4 = t4;
-                            w_trunc = cnt > 5;
-                            w_built = true;
+#pragma unroll
+                            for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                                const int m = __reduce_max_sync(kFull, t0);
+                                gw[r] = m;
+                                if (t0 == m) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = 0; }
+                            }
+                            gw_valid = true;
                         }
-                        int h0 = wt0, h1 = wt1, h2 = wt2, h3 = wt3, h4 = wt4;
-                        bool dry = false;
-                        nwin = 0;
 #pragma unroll
                         for (int r = 0; r < BR_MAX_RMAX; ++r) {
-                            win[r] = 0;
-                            if (r < a.R_max && r < n_left) {
-                                dry = dry || (h0 == 0 && w_trunc);
-                                const int m = __reduce_max_sync(kFull, h0);
-                                win[r] = m;
-                                if (m > 0) nwin = r + 1;
-                                if (h0 == m) { h0 = h1; h1 = h2; h2 = h3; h3 = h4; h4 = 0; }
-                            }
+                            win[r] = (r < a.R_max && r < n_left) ? gw[r] : 0;
+                            if (win[r] > 0) nwin = r + 1;
                         }
-                        if (!w_keep) { w_built = false; break; }
-                        if (!__any_sync(kFull, dry)) break;
-                        w_built = false;
+                    } else {
+                        // Eq. 2 kernels keep every lane's sorted candidates across pops and merge the
+                        // heads.  A list that runs dry although its lane holds more keys (possible only
+                        // after several admissions from one lane) forces a rebuild.
+#pragma unroll 1
+                        for (int attempt = 0; attempt < 2; ++attempt) {
+                            if (!w_built) {
+                                int t0 = 0, t1 = 0, t2 = 0, t3 = 0, t4 = 0, cnt = 0;
+#pragma unroll 4
+                                for (int t = 0; t < n_tiles; ++t) {
+                                    const int idx = (t << 5) + lane;
+                                    int x = idx < n_w ? q_key[idx] : 0;
+                                    cnt += x > 0;
+                                    int y;
+                                    y = max(t0, x); x = min(t0, x); t0 = y;
+                                    y = max(t1, x); x = min(t1, x); t1 = y;
+                                    y = max(t2, x); x = min(t2, x); t2 = y;
+                                    y = max(t3, x); x = min(t3, x); t3 = y;
+                                    t4 = max(t4, x);
+                                }
+                                wt0 = t0; wt1 = t1; wt2 = t2; wt3 = t3; wt4 = t4;
+                                w_trunc = cnt > 5;
+                                w_built = true;
+                            }
+                            int h0 = wt0, h1 = wt1, h2 = wt2, h3 = wt3, h4 = wt4;
+                            bool dry = false;
+                            nwin = 0;
+#pragma unroll
+                            for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                                win[r] = 0;
+                                if (r < a.R_max && r < n_left) {
+                                    dry = dry || (h0 == 0 && w_trunc);
+                                    const int m = __reduce_max_sync(kFull, h0);
+                                    win[r] = m;
+                                    if (m > 0) nwin = r + 1;
+                                    if (h0 == m) { h0 = h1; h1 = h2; h2 = h3; h3 = h4; h4 = 0; }
+                                }
+                            }
+                            if (!__any_sync(kFull, dry)) break;
+                            w_built = false;
+                        }
                     }
                     // subsets of the window: lane = mask, lowest mask on ties
                     const int lim = min(mc, a.R_max);
