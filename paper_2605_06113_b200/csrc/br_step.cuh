@@ -797,7 +797,14 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         fk = sc.key(a, delta);
                     }
                     long long wk;
-                    const int best_mask = warp_argmax_lane(fk, 31u - (unsigned)lane, wk);
+                    int best_mask;
+                    if (!FP) {                          // Eq. 1 scores fit 32 bits
+                        int wk32;
+                        best_mask = warp_argmax_lane32(fk == kNoKey ? kEmpty : (int)fk, 31u - (unsigned)lane, wk32);
+                        wk = wk32 == kEmpty ? kNoKey : (long long)wk32;
+                    } else {
+                        best_mask = warp_argmax_lane(fk, 31u - (unsigned)lane, wk);
+                    }
                     if (wk == kNoKey) { status |= BR_ST_ITER_CAP; break; }
                     if (wk <= 0) {
                         // starvation guard: least-bad single request of all of R_wait
