@@ -68,6 +68,18 @@ def recorded_traffic(workload: str):
     return None
 
 
+def recorded_instructions(workload: str):
+    """Warp instructions per launch from the same ncu capture (None if the kernel changed)."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        rec = json.load(open(p))
+        if rec.get("kernel_source_hash") == kernel_source_hash():
+            return rec.get("warp_instructions_per_launch", {}).get(workload)
+    except Exception:
+        pass
+    return None
+
+
 def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
     """Bytes one instance-step has to move once: running-request state in, queue in,
     assignments out, per-worker state in and out, slot edits."""
@@ -322,12 +334,28 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
         torch.cuda.synchronize()
         host_us.append(1e6 * (time.perf_counter() - t0))
         dev_us.append(1e3 * e0.elapsed_time(e1))
+    # per-phase split of the step (the kernel's own cycle counters; the paper splits its dispatcher
+    # the same way: preparation / Stage 1 / Stage 2), averaged over the next 200 steps
+    out["phase_cycles"] = torch.zeros((1, 1, 8), dtype=torch.int32, device=device)
+    acc = np.zeros(8)
+    n_ph = 200
+    for k in range(steps, steps + n_ph):
+        if cfg.H > 0:
+            wlm.term_probs_torch(wl, k, device, seeds_t=seeds_t, tab_t=tab_t, out=probs)
+        r.step(st, out, probs)
+        torch.cuda.synchronize()
+        acc += out["phase_cycles"][0, 0].cpu().numpy()
+    mhz = float(torch.cuda.get_device_properties(device).clock_rate) / 1e3 if hasattr(
+        torch.cuda.get_device_properties(device), "clock_rate") else 1965.0
+    names = ["arrive", "predict", "stage1", "stage2", "record_compact", "advance", "prologue", "kernel_total"]
+    phases = {n: float(acc[i] / n_ph / mhz) for i, n in enumerate(names)}
     r.close()
     h = np.array(host_us[20:]); d = np.array(dev_us[20:])
     return {"workload": cfg_name, "G": cfg.G, "W": cfg.W, "H": cfg.H, "steps": steps,
             "host_p50_us": float(np.percentile(h, 50)), "host_p95_us": float(np.percentile(h, 95)),
             "host_p99_us": float(np.percentile(h, 99)), "device_p50_us": float(np.percentile(d, 50)),
-            "device_p99_us": float(np.percentile(d, 99))}
+            "device_p99_us": float(np.percentile(d, 99)),
+            "phase_us_at_max_clock": phases}
 
 
 def run_ours(args):
@@ -362,6 +390,16 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": abytes,
                 "kernel": "br_step_kernel<false,0,1,2>" if wname == "c3" else "br_step_kernel<true,8,2,1>"}
 
+    winst = recorded_instructions(wname)
+    if winst:
+        # what actually binds the step: instruction issue.  Peak = 148 SMs x 4 schedulers x 1 warp
+        # instruction per clock at the SM clock sampled during the run.
+        clk = (clocks.get("sm_mhz") or 1965.0) * 1e6
+        peak_issue = 148 * 4 * clk
+        ach = winst / (ms * 1e-3 / args.steps)
+        roofline["issue"] = {"bound": "alu", "achieved": ach / 1e9, "peak": peak_issue / 1e9,
+                             "unit": "G warp-instructions/s", "frac": ach / peak_issue,
+                             "warp_instructions_per_launch": winst}
     line = {
         "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
         "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

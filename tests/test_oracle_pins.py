@@ -551,3 +551,32 @@ def test_hazard_decision_has_probability_thr_over_2_32():
         for v in vs:
             for w in ws:
                 assert oracle.term_decision(v, w, thr) == (((v << 16) | w) < thr)
+
+
+def test_best_subset_agrees_with_reachable_sums_and_two_probe_rule():
+    """The Stage-2 subproblem depends on Q only through Delta(Q) (Appendix 'Bit-set subset
+    selection'): a second, independent solver that enumerates the reachable sums per cardinality
+    must find the same optimum, and for BR-0 the optimum is one of two probes: the largest
+    reachable sum at or below the margin, or the smallest one above it."""
+    rng = np.random.default_rng(47)
+    for _ in range(300):
+        G = int(rng.integers(2, 33)); nw = int(rng.integers(1, 6)); lim = int(rng.integers(1, 6))
+        win = sorted((int(x) for x in rng.integers(1, 400, nw)), reverse=True)
+        m = int(rng.integers(0, 900))
+        reach = [set() for _ in range(lim + 1)]        # reach[j] = sums of exactly j window entries
+        reach[0].add(0)
+        for s in win:
+            for j in range(min(lim, nw), 0, -1):
+                reach[j] |= {x + s for x in reach[j - 1]}
+        sums = sorted(set().union(*reach[1:]))
+        mask, f = oracle.best_subset(0, G, 0, 1.0, float(G), 1.0, [m], win, lim)
+        assert f == max(oracle.f_br0(G, d, m) for d in sums)
+        below = [d for d in sums if d <= m]
+        above = [d for d in sums if d > m]
+        probes = ([max(below)] if below else []) + ([min(above)] if above else [])
+        assert f == max(oracle.f_br0(G, d, m) for d in probes)
+        assert sum(win[j] for j in range(nw) if mask >> j & 1) in sums
+        # horizon score: same statement with the reachable sums (no two-probe shortcut)
+        H = int(rng.integers(1, 5)); mh = rng.integers(0, 900, H + 1)
+        mask, f = oracle.best_subset(1, G, H, 1.0, 4.0, 0.5, mh, win, lim)
+        assert f == max(oracle.f_brh(H, 1.0, 4.0, 0.5, d, mh) for d in sums)
