@@ -249,7 +249,7 @@ class RotatingSets:
             big = self.sets[0]["wl"]
             big_tab = wlm.Workload(cfg=big.cfg, seeds=big.seeds, len_tab=big.len_tab, beta_tab=big.beta_tab,
                                    arr_cdf=table, arr_period=big.arr_period,
-                                   arr_inst_stride=big.arr_inst_stride, hazard_thr=big.hazard_thr,
+                                   arr_inst_stride=big.arr_inst_stride, term_cdf=big.term_cdf,
                                    state=big.state)
             self.router = Router(big_tab, device=device, threads=threads, **params)
         # all sets share one allocation per array so that `first_instance` selects the set

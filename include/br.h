@@ -28,7 +28,7 @@
 extern "C" {
 #endif
 
-#define BR_VERSION 100
+#define BR_VERSION 101
 
 /* status codes returned by every entry point */
 #define BR_OK        0
@@ -69,10 +69,13 @@ typedef struct {
     float   gate;           /* confidence gate on p_fin; < 0 -> 0.5                          */
     float   c_floor;        /* lower bound of c_hat; < 0 -> 1                                */
     int32_t score_mode;     /* 0: Eq. 1 in integers (needs H == 0); 1: Eq. 2 in fp64; < 0 -> 0 if H == 0 else 1 */
-    int32_t term_mode;      /* 0: requests never end; 1: end with probability hazard_thr / 2^32 per step
-                               (16 Philox bits per slot, 16 more when they tie with the threshold);
-                               2: end when a 24-bit Philox uniform < term_probs[slot][0]     */
-    uint32_t hazard_thr;
+    int32_t term_mode;      /* 0: requests never end; 1: every slot ends with the same probability p per
+                               step, independently (term_cdf); 2: end when a 24-bit Philox uniform <
+                               term_probs[slot][0]                                              */
+    const uint32_t *term_cdf; /* device [B], term_mode 1: term_cdf[j] = floor(2^32 (1 - (1-p)^(j+1))), the
+                               CDF of the number of slots skipped before the next ending one.  Per
+                               worker and step the ending slots are walked by these gaps: draw t is
+                               word t % 4 of the Philox block (k, g, TERM, t / 4), gap = #{j : u >= term_cdf[j]} */
     const uint32_t *arr_cdf;/* device [rows][arr_len] Poisson CDF thresholds; the row for instance i
                                at step k is i * arr_inst_stride + k % arr_period; NULL -> no arrivals */
     int32_t arr_len, arr_period, arr_inst_stride;

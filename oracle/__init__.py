@@ -35,7 +35,7 @@ class OrcParams(C.Structure):
         ("R_max", C.c_int32), ("S_greedy", C.c_int32),
         ("alpha", C.c_double), ("beta", C.c_double), ("gamma", C.c_double),
         ("delta_T", C.c_int32), ("gate", C.c_float), ("c_floor", C.c_float),
-        ("score_mode", C.c_int32), ("term_mode", C.c_int32), ("hazard_thr", C.c_uint32),
+        ("score_mode", C.c_int32), ("term_mode", C.c_int32), ("term_cdf", C.c_void_p),
         ("arr_cdf", C.c_void_p), ("arr_len", C.c_int32), ("arr_period", C.c_int32),
         ("len_tab", C.c_void_p), ("len_tab_log2", C.c_int32),
         ("burst_every", C.c_int32), ("burst_size", C.c_int32), ("router", C.c_int32),
@@ -59,8 +59,8 @@ def lib():
         L.orc_projection.argtypes = [C.c_void_p] + [C.c_void_p] * 3
         L.orc_predict_only.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_philox4x32_10.argtypes = [C.c_void_p] * 3
-        L.orc_term_decision.restype = C.c_int
-        L.orc_term_decision.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32]
+        L.orc_term_gap.restype = C.c_int
+        L.orc_term_gap.argtypes = [C.c_void_p, C.c_int32, C.c_uint32]
         L.orc_f_br0.restype = C.c_int64
         L.orc_f_br0.argtypes = [C.c_int32, C.c_int64, C.c_int64]
         L.orc_f_brh.restype = C.c_double
@@ -94,8 +94,10 @@ def philox4x32_10(ctr, key) -> np.ndarray:
     return out
 
 
-def term_decision(v16: int, w16: int, thr: int) -> bool:
-    return bool(lib().orc_term_decision(v16, w16, thr))
+def term_gap(term_cdf, u: int) -> int:
+    """Slots skipped before the next ending one, from one uniform 32-bit word."""
+    t = np.ascontiguousarray(term_cdf, dtype=np.uint32)
+    return int(lib().orc_term_gap(_p(t), len(t), int(u)))
 
 
 def f_br0(G: int, delta: int, m: int) -> int:
@@ -150,13 +152,16 @@ class Instance:
 
     def __init__(self, *, G, H, B, W, R_max=4, S_greedy=None, alpha=1.0, beta=None, gamma=1.0,
                  delta_T=None, gate=0.5, c_floor=1.0, score_mode=None, term_mode=0,
-                 hazard_thr=0, arr_rows=None, len_tab=None, burst_every=0, burst_size=0,
+                 term_cdf=None, arr_rows=None, len_tab=None, burst_every=0, burst_size=0,
                  router=0, seed=0):
         self.G, self.H, self.B, self.W = G, H, B, W
         self._arr = np.ascontiguousarray(
             arr_rows if arr_rows is not None else np.full((1, 1), 0xFFFFFFFF), dtype=np.uint32)
         self._len = np.ascontiguousarray(
             len_tab if len_tab is not None else np.ones(2, dtype=np.int32), dtype=np.int32)
+        self._term = np.ascontiguousarray(
+            term_cdf if term_cdf is not None else np.zeros(B, dtype=np.uint32), dtype=np.uint32)
+        assert self._term.shape == (B,)
         log2 = int(self._len.size).bit_length() - 1
         assert 1 << log2 == self._len.size
         p = OrcParams(
@@ -164,7 +169,7 @@ class Instance:
             alpha=alpha, beta=float(G) if beta is None else beta, gamma=gamma,
             delta_T=max(1, H // 2) if delta_T is None else delta_T, gate=gate, c_floor=c_floor,
             score_mode=(0 if H == 0 else 1) if score_mode is None else score_mode,
-            term_mode=term_mode, hazard_thr=hazard_thr,
+            term_mode=term_mode, term_cdf=self._term.ctypes.data,
             arr_cdf=self._arr.ctypes.data, arr_len=self._arr.shape[1],
             arr_period=self._arr.shape[0], len_tab=self._len.ctypes.data, len_tab_log2=log2,
             burst_every=burst_every, burst_size=burst_size, router=router)
@@ -243,7 +248,7 @@ def instance_from_workload(wl, inst: int, router: int = 0, **overrides) -> Insta
     kw = dict(G=cfg.G, H=cfg.H, B=cfg.B, W=cfg.W, R_max=cfg.R_max, S_greedy=cfg.S_greedy,
               alpha=cfg.alpha, beta=cfg.beta, gamma=cfg.gamma, delta_T=cfg.delta_T,
               gate=cfg.gate, c_floor=cfg.c_floor, score_mode=cfg.score_mode,
-              term_mode=cfg.term_mode, hazard_thr=wl.hazard_thr, arr_rows=wl.arr_rows_for(inst),
+              term_mode=cfg.term_mode, term_cdf=wl.term_cdf, arr_rows=wl.arr_rows_for(inst),
               len_tab=wl.len_tab, burst_every=cfg.burst_every, burst_size=cfg.burst_size,
               router=router, seed=int(wl.seeds[inst]))
     if cfg.score_mode == 0:

@@ -41,7 +41,7 @@ typedef struct {
     float   gate, c_floor;
     int32_t score_mode;          /* 0: Eq. 1 in integers; 1: Eq. 2 in fp64          */
     int32_t term_mode;           /* 0 none; 1 constant hazard; 2 Bernoulli(probs[.][0]) */
-    uint32_t hazard_thr;
+    const uint32_t *term_cdf;    /* [B] gap thresholds of the constant hazard (term_mode 1) */
     const uint32_t *arr_cdf;     /* [arr_period][arr_len] rows for this instance    */
     int32_t arr_len, arr_period;
     const int32_t *len_tab;
@@ -98,7 +98,7 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2, STREAM_TERM_REFINE = 3 };
+enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2 };
 
 static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
 {
@@ -111,34 +111,40 @@ static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
 }
 
 /*
- * Constant-hazard termination of the request in slot a at step k: a Bernoulli event of
- * probability thr / 2^32 realised from 16 + 16 Philox bits.  The first 16 bits v are
- * half j % 2 of word j / 2 (j = a % 8) of the block with counter (k, a / 8, TERM, 0);
- * they decide unless v equals the high half of thr, in which case the low 16 bits of
- * word 0 of the block (k, a, TERM_REFINE, 0) are compared with the low half of thr.
+ * Constant-hazard terminations of worker g at step k (term_mode 1).  Every slot of the
+ * worker ends with the same probability p, independently; the slots that end are found by
+ * their gaps: the number of slots skipped before the next ending one is geometric, and
+ * term_cdf[j] = floor(2^32 P(gap <= j)) = floor(2^32 (1 - (1 - p)^(j+1))) is its CDF on the
+ * 32-bit scale, so a uniform word u gives gap = #{j < B : u >= term_cdf[j]} (B = none left).
+ * Draw t of the worker is word t % 4 of the Philox block with counter (k, g, TERM, t / 4).
+ * fin[b] is set for every slot b of the worker that ends, occupied or not.
  * READING: the paper fixes only the per-step probability (Section 2.2 leaves o_i latent);
- * the bit recipe is this workload's, chosen so that one Philox block serves 8 slots.
+ * independent Bernoulli(p) slots and geometric gaps between successes are the same law.
  */
-int orc_term_decision(uint32_t v16, uint32_t w16, uint32_t thr)
+int orc_term_gap(const uint32_t *term_cdf, int32_t B, uint32_t u)
 {
-    uint32_t hi = thr >> 16, lo = thr & 0xFFFFu;
-    return v16 < hi || (v16 == hi && w16 < lo);
+    int gap = 0;
+    for (int j = 0; j < B; ++j) if (u >= term_cdf[j]) ++gap;
+    return gap;
 }
 
-static int hazard_fin(const orc_inst *s, uint32_t a)
+static void hazard_fin(const orc_inst *s, int g, uint8_t *fin)
 {
+    const orc_params *p = &s->p;
     uint32_t key[2] = { (uint32_t)s->seed, (uint32_t)(s->seed >> 32) };
-    uint32_t ctr[4] = { (uint32_t)s->k, a >> 3, STREAM_TERM, 0u };
-    uint32_t out[4], ref[4];
-    orc_philox4x32_10(ctr, key, out);
-    uint32_t j = a & 7u;
-    uint32_t v16 = (out[j >> 1] >> (16u * (j & 1u))) & 0xFFFFu;
-    ref[0] = 0u;
-    if (v16 == (s->p.hazard_thr >> 16)) {          /* the second draw matters only on equality */
-        uint32_t ctr2[4] = { (uint32_t)s->k, a, STREAM_TERM_REFINE, 0u };
-        orc_philox4x32_10(ctr2, key, ref);
+    uint32_t out[4];
+    int pos = 0;
+    for (int b = 0; b < p->B; ++b) fin[b] = 0;
+    for (uint32_t t = 0; pos < p->B; ++t) {
+        if ((t & 3u) == 0u) {
+            uint32_t ctr[4] = { (uint32_t)s->k, (uint32_t)g, STREAM_TERM, t >> 2 };
+            orc_philox4x32_10(ctr, key, out);
+        }
+        int slot = pos + orc_term_gap(p->term_cdf, p->B, out[t & 3u]);
+        if (slot >= p->B) break;
+        fin[slot] = 1;
+        pos = slot + 1;
     }
-    return orc_term_decision(v16, ref[0] & 0xFFFFu, s->p.hazard_thr);
 }
 
 /* ------------------------------------------------------------------ */
@@ -547,8 +553,6 @@ void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
               int64_t *trace, double *fscore)
 {
     const orc_params *p = &s->p;
-    int A = p->G * p->B;
-
     arrive(s);
     predict(s, probs);
     project(s);
@@ -584,18 +588,24 @@ void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
 
     /* ADVANCE: every running request, the just-admitted ones included, either
      * finishes at the end of this step or grows by one token */
-    for (int a = 0; a < A; ++a) {
-        if (!s->occ[a]) continue;
-        int fin = 0;
-        if (p->term_mode == 1) {
-            fin = hazard_fin(s, (uint32_t)a);
-        } else if (p->term_mode == 2) {
-            uint32_t u = draw(s, (uint32_t)a, STREAM_TERM) >> 8;       /* 24 bits */
-            fin = ((float)u * 5.9604644775390625e-8f) < probs[(size_t)a * p->H];
+    uint8_t *fin_g = (uint8_t *)malloc((size_t)p->B);
+    for (int g = 0; g < p->G; ++g) {
+        if (p->term_mode == 1) hazard_fin(s, g, fin_g);
+        for (int b = 0; b < p->B; ++b) {
+            int a = g * p->B + b;
+            if (!s->occ[a]) continue;
+            int fin = 0;
+            if (p->term_mode == 1) {
+                fin = fin_g[b];
+            } else if (p->term_mode == 2) {
+                uint32_t u = draw(s, (uint32_t)a, STREAM_TERM) >> 8;       /* 24 bits */
+                fin = ((float)u * 5.9604644775390625e-8f) < probs[(size_t)a * p->H];
+            }
+            if (fin) { s->occ[a] = 0; s->cur[a] = 0; }
+            else s->cur[a] += 1;
         }
-        if (fin) { s->occ[a] = 0; s->cur[a] = 0; }
-        else s->cur[a] += 1;
     }
+    free(fin_g);
     s->k += 1;
 }
 

@@ -24,7 +24,7 @@ class BrParams(C.Structure):
         ("B", C.c_int32), ("W", C.c_int32), ("R_max", C.c_int32), ("S_greedy", C.c_int32),
         ("alpha", C.c_double), ("beta", C.c_double), ("gamma", C.c_double),
         ("delta_T", C.c_int32), ("gate", C.c_float), ("c_floor", C.c_float),
-        ("score_mode", C.c_int32), ("term_mode", C.c_int32), ("hazard_thr", C.c_uint32),
+        ("score_mode", C.c_int32), ("term_mode", C.c_int32), ("term_cdf", C.c_void_p),
         ("arr_cdf", C.c_void_p), ("arr_len", C.c_int32), ("arr_period", C.c_int32),
         ("arr_inst_stride", C.c_int32),
         ("len_tab", C.c_void_p), ("len_tab_log2", C.c_int32),
@@ -130,10 +130,11 @@ class Router:
         self.device = torch.device(device)
         self.len_tab = _to_torch(wl.len_tab, self.device)
         self.arr_cdf = _to_torch(wl.arr_cdf, self.device)
+        self.term_cdf = _to_torch(wl.term_cdf, self.device)
         p = BrParams(
             B=cfg.B, W=cfg.W, R_max=cfg.R_max, S_greedy=cfg.S_greedy, alpha=cfg.alpha,
             beta=cfg.beta, gamma=cfg.gamma, delta_T=cfg.delta_T, gate=cfg.gate, c_floor=cfg.c_floor,
-            score_mode=cfg.score_mode, term_mode=cfg.term_mode, hazard_thr=wl.hazard_thr,
+            score_mode=cfg.score_mode, term_mode=cfg.term_mode, term_cdf=self.term_cdf.data_ptr(),
             arr_cdf=self.arr_cdf.data_ptr(), arr_len=wl.arr_cdf.shape[1], arr_period=wl.arr_period,
             arr_inst_stride=wl.arr_inst_stride, len_tab=self.len_tab.data_ptr(),
             len_tab_log2=int(wl.len_tab.size).bit_length() - 1, burst_every=cfg.burst_every,

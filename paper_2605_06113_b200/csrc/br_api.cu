@@ -159,6 +159,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     if (p.score_mode < 0) p.score_mode = (H == 0) ? 0 : 1;
     if (p.score_mode > 1 || (p.score_mode == 0 && H != 0)) return BR_EINVAL;
     if (p.term_mode < 0 || p.term_mode > 2 || (p.term_mode == 2 && H == 0)) return BR_EINVAL;
+    if (p.term_mode == 1 && !p.term_cdf) return BR_EINVAL;
     if (p.arr_cdf) {
         if (p.arr_len < 1 || p.arr_period < 1 || p.arr_inst_stride < 0 || !p.len_tab) return BR_EINVAL;
         if (p.len_tab_log2 < 0 || p.len_tab_log2 > 24) return BR_EINVAL;
@@ -204,7 +205,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     a.wl = wl;
     a.magic_B = (uint32_t)(((1ull << 32) + (unsigned)p.B - 1) / (unsigned)p.B);
     a.delta_T = p.delta_T; a.gate = p.gate; a.c_floor = p.c_floor;
-    a.term_mode = p.term_mode; a.hazard_thr = p.hazard_thr;
+    a.term_mode = p.term_mode; a.term_cdf = p.term_cdf;
     a.arr_cdf = p.arr_cdf; a.arr_len = p.arr_len; a.arr_period = p.arr_period;
     a.arr_inst_stride = p.arr_inst_stride;
     a.len_tab = p.len_tab; a.len_shift = 32 - p.len_tab_log2;

@@ -11,7 +11,7 @@ constexpr int32_t kEmpty = INT32_MIN;
 constexpr long long kNoKey = (long long)0x8000000000000000ull;
 constexpr int kNoIdx = 0x7FFFFFFF;
 
-enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2, kStreamTermRefine = 3 };
+enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2 };
 
 // Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0, k1).
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

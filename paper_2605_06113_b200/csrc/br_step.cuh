@@ -27,7 +27,7 @@ struct StepArgs {
     int32_t delta_T;
     float gate, c_floor;
     int32_t term_mode;
-    uint32_t hazard_thr;
+    const uint32_t *term_cdf;   // [B] gap thresholds of the constant hazard
     const uint32_t *arr_cdf;
     int32_t arr_len, arr_period, arr_inst_stride;
     const int32_t *len_tab;
@@ -53,7 +53,7 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     n += 8 * (size_t)G * occ_words * 2;          // occ, end_mask
     n += 4 * (size_t)G * (H + 1) * 2;            // Lh_s, Ch_s (PREDICT buckets: load sums, counts)
     n += 4 * (size_t)G;                          // sub_load
-    n += 2 * (((size_t)G * B / 8 + 15) & ~(size_t)15);   // fin_b, eq_b
+    n += 8 * (size_t)G * occ_words;              // fin_w
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
     if (H > 0) n += 2 * (size_t)G * B;           // refresh_list
     return (n + 15) & ~(size_t)15;
@@ -119,10 +119,33 @@ __device__ __forceinline__ int warp_argmax_lane32(int key, unsigned tie, int &wk
     return __ffs(who) - 1;
 }
 
-// nonzero iff some 16-bit field of x is below n (n <= 0x8000)
-__device__ __forceinline__ unsigned hasless16(unsigned x, unsigned n)
+// Slots of worker g that end at step k under the constant hazard, as bit masks of 64 slots each.
+// Slots end independently with one probability, so the ending ones are walked by their gaps:
+// cdf[j] = floor(2^32 P(gap <= j)), draw t is word t % 4 of the Philox block (k, g, TERM, t / 4),
+// and a word u skips gap = #{j : u >= cdf[j]} slots (cdf ascends: the first j with u < cdf[j]).
+__device__ __forceinline__ void draw_ending(const uint32_t *__restrict__ cdf, int B, int OW, uint32_t k,
+                                            uint32_t g, uint32_t key0, uint32_t key1,
+                                            unsigned long long *out)
 {
-    return (x - 0x00010001u * n) & ~x & 0x80008000u;
+    for (int w = 0; w < OW; ++w) out[w] = 0ull;
+    int pos = 0;
+    uint4 r = philox4x32_10(k, g, kStreamTerm, 0u, key0, key1);
+#pragma unroll 1
+    for (unsigned t = 0; t < (unsigned)B; ++t) {          // every draw moves pos forward
+        if (t != 0u && (t & 3u) == 0u) r = philox4x32_10(k, g, kStreamTerm, t >> 2, key0, key1);
+        const uint32_t u = word_of(r, t & 3u);
+        const int room = B - pos;
+        if (u >= __ldg(cdf + room - 1)) break;            // the gap reaches past the last slot
+        int lo = 0, hi = room - 1;                        // u < cdf[hi]
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (u < __ldg(cdf + mid)) hi = mid; else lo = mid + 1;
+        }
+        const int slot = pos + lo;
+        out[slot >> 6] |= 1ull << (slot & 63);
+        pos = slot + 1;
+        if (pos >= B) break;
+    }
 }
 
 constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
@@ -153,7 +176,6 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     const int WL = a.wl;
     const unsigned posmask = (1u << WL) - 1u;
     const int inst = a.first_instance + blockIdx.x * per_block + in_block;
-    const unsigned thr_hi = a.hazard_thr >> 16, thr_lo = a.hazard_thr & 0xFFFFu;
     const unsigned t_entry = (unsigned)clock64();
 
     // ---- shared-memory carve-up (sizes match step_smem_bytes) ----
@@ -161,9 +183,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned *q_id = reinterpret_cast<unsigned *>(q_key + W);                       // [W]
     unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_id + W);     // [G][OW]
     unsigned long long *end_mask = occ + (size_t)G * OW;                            // [G][OW]
-    unsigned char *fin_b = reinterpret_cast<unsigned char *>(end_mask + (size_t)G * OW);   // [A/8], 8-byte aligned
-    unsigned char *eq_b = fin_b + (((size_t)A8 + 15) & ~(size_t)15);                // [A/8]
-    unsigned *Lh_s = reinterpret_cast<unsigned *>(eq_b + (((size_t)A8 + 15) & ~(size_t)15));   // [G][H1]
+    unsigned long long *fin_w = end_mask + (size_t)G * OW;                          // [G][OW] slots whose draw says "ends"
+    unsigned *Lh_s = reinterpret_cast<unsigned *>(fin_w + (size_t)G * OW);          // [G][H1]
     unsigned *Ch_s = Lh_s + (size_t)G * H1;                                         // [G][H1]
     unsigned *sub_load = Ch_s + (size_t)G * H1;                                     // [G]
     unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
@@ -214,7 +235,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         if (i1 < W) fetch_queue(i1);
     }
     for (int i = (2 * NT + tid) * 4; i < n_w; i += NT * 4) fetch_queue(i);
-    for (int i = tid; i < G * OW; i += NT) occ[i] = g_occ[i];
+    for (int i = tid; i < G * OW; i += NT) { occ[i] = g_occ[i]; fin_w[i] = 0ull; }
     for (int i = tid; i < 2 * G * H1; i += NT) Lh_s[i] = 0u;      // Lh_s and Ch_s are adjacent
     for (int i = tid; i < G; i += NT) sub_load[i] = 0u;
 
@@ -240,35 +261,11 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     inst_sync();
     if (prologue_status) atomicOr(&scal[5], prologue_status);
 
-    // Philox words of the step's constant-hazard terminations: per 8-slot group one byte of
-    // "first 16 bits below the high half of the threshold" and one of "equal to it"
-    auto draw_terms = [&](int first, int stride) {
+    // this step's constant-hazard draws of workers first, first + stride, ...
+    auto draw_fin = [&](int first, int stride) {
 #pragma unroll 1
-        for (int q_base = first; q_base < A8; q_base += 4 * stride) {
-            // four independent Philox blocks in flight per thread
-            uint4 r[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                r[u] = philox4x32_10((uint32_t)k, (uint32_t)(q_base + u * stride), kStreamTerm, 0u, key0, key1);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int q8 = q_base + u * stride;
-                unsigned fb = 0, eb = 0;
-                const unsigned wv[4] = {r[u].x, r[u].y, r[u].z, r[u].w};
-                unsigned any = 1u;
-                if (thr_hi < 0x8000u)       // smallest 16-bit draw of the block against the threshold
-                    any = hasless16(__vminu2(__vminu2(wv[0], wv[1]), __vminu2(wv[2], wv[3])), thr_hi + 1);
-                if (any) {          // rare: some 16-bit draw is at or below the high half of the threshold
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const unsigned lo16 = wv[w] & 0xFFFFu, hi16 = wv[w] >> 16;
-                        fb |= ((lo16 < thr_hi ? 1u : 0u) | (hi16 < thr_hi ? 2u : 0u)) << (2 * w);
-                        eb |= ((lo16 == thr_hi ? 1u : 0u) | (hi16 == thr_hi ? 2u : 0u)) << (2 * w);
-                    }
-                }
-                if (q8 < A8) { fin_b[q8] = (unsigned char)fb; eq_b[q8] = (unsigned char)eb; }
-            }
-        }
+        for (int g = first; g < G; g += stride)
+            draw_ending(a.term_cdf, B, OW, (uint32_t)k, (uint32_t)g, key0, key1, fin_w + (size_t)g * OW);
     };
 
     // Per worker word: which running requests end at this step (occupancy & termination draws).
@@ -279,28 +276,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         for (int idx = tid; idx < G * OW; idx += NT) {
             const int g = idx / OW, x = idx - g * OW;
             const unsigned long long occw = occ[idx];
-            unsigned long long finw = 0ull, eqw = 0ull;
-            if (term_mode != 0 && occw) {
-                const int b0 = g * (B >> 3) + 8 * x;
-                const int nb = min(8, (B >> 3) - 8 * x);
-                if (nb == 8 && (b0 & 7) == 0) {
-                    finw = *reinterpret_cast<const unsigned long long *>(fin_b + b0);
-                    eqw = *reinterpret_cast<const unsigned long long *>(eq_b + b0);
-                } else {
-                    for (int b = 0; b < nb; ++b) {
-                        finw |= (unsigned long long)fin_b[b0 + b] << (8 * b);
-                        eqw |= (unsigned long long)eq_b[b0 + b] << (8 * b);
-                    }
-                }
-                unsigned long long cand = occw & eqw & ~finw;
-                while (cand) {                                       // first 16 bits tied: 16 more decide
-                    const int j = __ffsll((long long)cand) - 1;
-                    cand &= cand - 1;
-                    const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)(g * B + 64 * x + j),
-                                                     kStreamTermRefine, 0u, key0, key1).x;
-                    if ((w & 0xFFFFu) < thr_lo) finw |= 1ull << j;
-                }
-            }
+            const unsigned long long finw = term_mode != 0 ? fin_w[idx] : 0ull;
             unsigned long long ended = occw & finw;
             end_mask[idx] = ended;
             while (ended) {
@@ -346,7 +322,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         const bool have_pre = (nwarps == 1 && term_mode == 1);
         int pend = 0, n_pre = 0;
         if (have_pre) {
-            draw_terms(tid, NT);
+            draw_fin(tid, NT);
             __syncwarp();
             scan_workers(true);
             __syncwarp();
@@ -846,7 +822,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             }
         } else if (term_mode == 1) {
             // warps 1.. draw this step's termination words while warp 0 routes
-            draw_terms(tid - 32, NT - 32);
+            draw_fin(tid - 32, NT - 32);
         }
         inst_sync();                                              // B2: admissions visible
 
@@ -869,13 +845,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 if (i < W) assign[i] = (gone && sa < A) ? sa : -1;
                 if (have_pre && gone && sa < A) {
                     // a request admitted at this step may also end at it
-                    unsigned fb = (fin_b[sa >> 3] >> (sa & 7)) & 1u;
-                    if (!fb && ((eq_b[sa >> 3] >> (sa & 7)) & 1u)) {
-                        const uint32_t w = philox4x32_10((uint32_t)k, (uint32_t)sa, kStreamTermRefine, 0u, key0, key1).x;
-                        fb = (w & 0xFFFFu) < thr_lo;
-                    }
-                    if (fb) {
-                        const int g = sa / B, slot = sa - g * B;
+                    const int g = (int)__umulhi((unsigned)sa, a.magic_B), slot = sa - g * B;
+                    if ((fin_w[g * OW + (slot >> 6)] >> (slot & 63)) & 1ull) {
                         atomicOr(&end_mask[g * OW + (slot >> 6)], 1ull << (slot & 63));
                         const int at = atomicAdd(&scal[6], 1);
                         if (at < kEndList) {
@@ -930,8 +901,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                             }
                         }
                     }
-                    fin_b[q8] = (unsigned char)fb;
-                    eq_b[q8] = 0;
+                    reinterpret_cast<unsigned char *>(fin_w + (size_t)g * OW)[slot0 >> 3] = (unsigned char)fb;
                 }
                 inst_sync();
             }

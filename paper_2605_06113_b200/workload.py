@@ -112,9 +112,20 @@ def poisson_thresholds(lam) -> np.ndarray:
     return np.minimum(t, 4294967295.0).astype(np.uint32)
 
 
-def hazard_threshold(p: float) -> int:
-    """u32 threshold: a uniform word u terminates the request iff u < thr."""
-    return int(min(4294967295, round(p * 4294967296.0)))
+def termination_gap_thresholds(p: float, B: int) -> np.ndarray:
+    """uint32 t[j] = min(2^32-1, floor(P(gap <= j) * 2^32)), j < B, for slots that end
+    independently with probability p each: the number of slots skipped before the next ending
+    one is geometric, P(gap <= j) = 1 - (1 - p)^(j+1).  A uniform 32-bit word u realises
+    gap = #{j : u >= t[j]}; gap = B means that no further slot of the worker ends.
+    """
+    j = np.arange(1, B + 1, dtype=np.float64)
+    if p <= 0.0:
+        cdf = np.zeros(B, dtype=np.float64)
+    elif p >= 1.0:
+        cdf = np.ones(B, dtype=np.float64)
+    else:
+        cdf = -np.expm1(j * math.log1p(-p))
+    return np.minimum(np.floor(cdf * 4294967296.0), 4294967295.0).astype(np.uint32)
 
 
 # --------------------------------------------------------------------------
@@ -206,7 +217,7 @@ class Workload:
     arr_cdf: np.ndarray           # uint32 [rows, ARR_LEN]
     arr_period: int
     arr_inst_stride: int          # row(inst, k) = inst * stride + k % period
-    hazard_thr: int
+    term_cdf: np.ndarray          # uint32 [B] gap thresholds of the constant hazard
     state: Dict[str, np.ndarray] = field(default_factory=dict)
 
     def arr_rows_for(self, inst: int) -> np.ndarray:
@@ -290,7 +301,7 @@ def make_workload(cfg: Config, n_instances: Optional[int] = None,
     )
     return Workload(cfg=cfg, seeds=seeds, len_tab=len_tab, beta_tab=btab, arr_cdf=arr,
                     arr_period=period, arr_inst_stride=stride,
-                    hazard_thr=hazard_threshold(cfg.hazard), state=state)
+                    term_cdf=termination_gap_thresholds(cfg.hazard, B), state=state)
 
 
 # --------------------------------------------------------------------------

@@ -27,14 +27,14 @@ def test_library_exports_every_declared_entry_point():
     for n in names:
         assert hasattr(L, n), n
     assert sorted(binding.EXPORTS) == names
-    assert L.br_version() == 100
+    assert L.br_version() == 101
     assert L.br_strerror(BR_OK) == b"ok"
     assert b"invalid" in L.br_strerror(BR_EINVAL)
 
 
 def _params(**kw):
     p = BrParams(B=64, W=256, R_max=0, S_greedy=-1, alpha=1.0, beta=14.67, gamma=0.64, delta_T=0,
-                 gate=-1.0, c_floor=-1.0, score_mode=-1, term_mode=1, hazard_thr=1000, arr_cdf=None,
+                 gate=-1.0, c_floor=-1.0, score_mode=-1, term_mode=1, term_cdf=0x1000, arr_cdf=None,
                  arr_len=0, arr_period=0, arr_inst_stride=0, len_tab=None, len_tab_log2=0,
                  burst_every=0, burst_size=0, s_max=131072, threads=0, inst_per_block=0)
     for k, v in kw.items():
@@ -58,7 +58,7 @@ def test_create_validates_sizes_and_ranges():
     for G, H, kw in [(0, 0, {}), (65, 0, {}), (32, 17, {}), (32, -1, {}), (32, 0, dict(B=12)),
                      (32, 0, dict(B=264)), (32, 0, dict(W=6)), (32, 0, dict(W=8192)),
                      (32, 0, dict(R_max=6)), (32, 4, dict(score_mode=0)), (32, 0, dict(term_mode=2)),
-                     (32, 0, dict(term_mode=3)), (32, 4, dict(gamma=0.0)), (32, 4, dict(gamma=1.5)),
+                     (32, 0, dict(term_mode=3)), (32, 0, dict(term_cdf=None)), (32, 4, dict(gamma=0.0)), (32, 4, dict(gamma=1.5)),
                      (32, 4, dict(alpha=-1.0)), (32, 0, dict(threads=48)), (32, 0, dict(threads=512)),
                      (32, 4, dict(delta_T=200))]:
         rc, h = _create(G, H, _params(**kw))

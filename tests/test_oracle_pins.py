@@ -512,7 +512,13 @@ def test_workload_tables_match_their_distributions():
         pmf = np.diff(np.concatenate([[0.0], thr / 2 ** 32]))
         mean = (np.arange(len(pmf)) * pmf).sum()
         assert abs(mean - lam) < 1e-3
-    assert wlm.hazard_threshold(1 / 500) == round(2 ** 32 / 500)
+    # gap thresholds of the constant hazard: P(gap = j) = p (1 - p)^j on the 32-bit scale
+    for p, B in [(1 / 500, 64), (1 / 400, 64), (0.05, 16), (0.5, 8)]:
+        t = wlm.termination_gap_thresholds(p, B).astype(np.float64)
+        assert t[0] == np.floor(p * 2 ** 32) and np.all(np.diff(t) >= 0)
+        pmf = np.diff(np.concatenate([[0.0], t])) / 2 ** 32
+        assert np.abs(pmf - p * (1 - p) ** np.arange(B)).max() < 2.0 ** -31
+    assert not wlm.termination_gap_thresholds(0.0, 8).any()
     # numpy and torch flavours of the counter mixer agree
     import torch
     seeds = np.arange(5, dtype=np.uint64) + np.uint64(2 ** 63 + 12345)
@@ -538,19 +544,67 @@ def test_stored_traces_are_reproduced():
         assert mg.run(name, steps) == want
 
 
-def test_hazard_decision_has_probability_thr_over_2_32():
-    """The 16 + 16 bit termination recipe fires exactly when the 32-bit word (v << 16 | w) is
-    below the threshold, so its probability is thr / 2^32."""
+def test_gap_of_a_word_is_the_count_of_thresholds_at_or_below_it():
+    """A uniform word u skips gap = #{j : u >= t[j]} slots: gap <= j exactly when u < t[j], so
+    P(gap <= j) = t[j] / 2^32 (the table is that CDF)."""
     rng = np.random.default_rng(41)
-    for thr in [0, 1, 0xFFFF, 0x10000, wlm.hazard_threshold(1 / 500), wlm.hazard_threshold(1 / 400),
-                0x7FFF8001, 0xFFFFFFFF]:
-        hi = thr >> 16
-        vs = sorted(set([0, 1, max(hi - 1, 0), hi, min(hi + 1, 0xFFFF), 0xFFFF] + [int(x) for x in rng.integers(0, 65536, 20)]))
-        ws = [0, 1, (thr & 0xFFFF), max((thr & 0xFFFF) - 1, 0), min((thr & 0xFFFF) + 1, 0xFFFF), 0xFFFF] + \
-             [int(x) for x in rng.integers(0, 65536, 20)]
-        for v in vs:
-            for w in ws:
-                assert oracle.term_decision(v, w, thr) == (((v << 16) | w) < thr)
+    for p, B in [(1 / 500, 64), (0.05, 16), (0.5, 8), (0.0, 8), (1.0, 8)]:
+        t = wlm.termination_gap_thresholds(p, B)
+        us = [0, 1, 0xFFFFFFFF] + [int(x) for x in rng.integers(0, 2 ** 32, 40)]
+        for j in range(B):
+            us += [int(t[j]), max(int(t[j]) - 1, 0), min(int(t[j]) + 1, 0xFFFFFFFF)]
+        for u in us:
+            gap = oracle.term_gap(t, u)
+            assert 0 <= gap <= B
+            for j in range(B):
+                assert (gap <= j) == (u < int(t[j]))
+
+
+def test_constant_hazard_slots_end_independently_with_probability_p():
+    """term_mode 1 realises independent Bernoulli(p) endings per slot and step (Section 2.2: each
+    running request ends with a fixed probability per step).  Checked on the law itself: per-slot
+    frequencies, the number ending per worker-step (binomial mean and variance), joint endings of
+    slot pairs, and the realised ending sets rebuilt from the Philox definition."""
+    G, B, p, steps = 3, 16, 0.08, 6000
+    t = wlm.termination_gap_thresholds(p, B)
+    seed = 0x1234_5678_9ABC_DEF1
+    o = oracle.Instance(G=G, H=0, B=B, W=4, term_mode=1, term_cdf=t, seed=seed)
+    base = np.full((G, B), 1000, dtype=np.int32)
+    ended = np.zeros((steps, G, B), dtype=bool)
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for k in range(steps):
+        o.set_state(k, 0, base - k, None, None, None, None, None, 0)     # all slots running again
+        o.step()
+        ended[k] = o.get_state()["act_base"] == EMPTY
+        if k < 40:
+            for g in range(G):       # the same sets from the definition: walk the gaps
+                want = np.zeros(B, dtype=bool); pos = 0; d = 0
+                while pos < B:
+                    u = _philox_py([k, g, 2, d // 4], key)[d % 4]
+                    slot = pos + int((u >= t.astype(np.int64)).sum())
+                    if slot >= B:
+                        break
+                    want[slot] = True; pos = slot + 1; d += 1
+                assert np.array_equal(ended[k, g], want)
+    n = steps * G
+    freq = ended.reshape(n, B).mean(0)
+    assert np.abs(freq - p).max() < 5 * np.sqrt(p * (1 - p) / n)
+    cnt = ended.reshape(n, B).sum(1)
+    assert abs(cnt.mean() - B * p) < 5 * np.sqrt(B * p * (1 - p) / n)
+    assert abs(cnt.var() - B * p * (1 - p)) < 0.1 * B * p * (1 - p)
+    e = ended.reshape(n, B)
+    for i, j in [(0, 1), (0, B - 1), (3, 4), (7, 12)]:
+        both = (e[:, i] & e[:, j]).mean()
+        assert abs(both - p * p) < 5 * np.sqrt(p * p / n)
+    # a slot that is free when the step ends is unaffected, an occupied one follows the same draw
+    o2 = oracle.Instance(G=G, H=0, B=B, W=4, term_mode=1, term_cdf=t, seed=seed)
+    k7 = int(np.argmax(ended[:, :, 1::2].sum((1, 2))))                  # a step where odd slots end
+    half = base - k7; half[:, ::2] = EMPTY
+    o2.set_state(k7, 0, half, None, None, None, None, None, 0)
+    o2.step()
+    got = o2.get_state()["act_base"] == EMPTY
+    assert ended[k7][:, 1::2].any()
+    assert np.array_equal(got[:, 1::2], ended[k7][:, 1::2]) and got[:, ::2].all()
 
 
 def test_best_subset_agrees_with_reachable_sums_and_two_probe_rule():
