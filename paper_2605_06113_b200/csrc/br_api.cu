@@ -8,6 +8,7 @@
 #include <new>
 
 #include "br_step.cuh"
+#include "br_small.cuh"
 #include "br_fscore.cuh"
 
 using br::StepArgs;
@@ -19,6 +20,7 @@ struct br_ctx {
     int threads;              // threads per instance for large batches
     int threads_small;        // ... for batches of a few instances (latency path)
     int inst_per_block;       // single-warp instances per thread block
+    bool small_ok;            // the fleet shape fits br_small_kernel
     size_t smem;
     // latency path
     cudaGraph_t graph;
@@ -102,6 +104,20 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.out = *out;
     // few instances: the launch is latency-bound, so spread each instance over more warps
     const int tpi = b->n_instances <= 64 ? ctx->threads_small : ctx->threads;
+    if (tpi == 32 && ctx->small_ok && !out->fscore && !out->phase_cycles) {
+        // BR-0 on a small fleet: the one-warp-per-instance kernel
+        int wpb = ctx->inst_per_block;
+        if (wpb > b->n_instances) wpb = b->n_instances;
+        const int nt4 = ctx->p.W <= 128 ? 1 : 2;
+        step_kernel_t kern = nt4 == 1 ? (ctx->p.R_max <= 4 ? br::br_small_kernel<1, 4> : br::br_small_kernel<1, 5>)
+                                      : (ctx->p.R_max <= 4 ? br::br_small_kernel<2, 4> : br::br_small_kernel<2, 5>);
+        a.tpi = 32;
+        const int blocks = (b->n_instances + wpb - 1) / wpb;
+        kern<<<blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * sizeof(int), stream>>>(a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
+        return BR_OK;
+    }
     const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles) ? (tpi == 32 ? 2 : 1) : 0;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
     // single-warp instances are packed several to a block
@@ -225,6 +241,11 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G;
     }
     ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
+    // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 256 waiting requests,
+    // arrivals served by one Philox call, and negative queue keys scoring below every waiting request
+    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 256 && p.term_mode != 2 &&
+                    p.burst_every == 0 && (!p.arr_cdf || p.arr_len <= 64) &&
+                    (long long)(G - 1) * p.s_max + 65536 < (1ll << (31 - wl));
     *out = ctx;
     return BR_OK;
 }

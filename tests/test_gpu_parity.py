@@ -96,3 +96,34 @@ def test_empty_and_saturated_edges():
     # empty fleet, long queue: first step admits min(S_tot, n_w)
     cfg = wlm.get_config("c1", init_active=0)
     run_parity(cfg, 1, 10)
+
+
+# ---- the one-warp-per-instance BR-0 kernel (G <= 32, B <= 64, W <= 256; threads=32 selects it) ----
+def test_small_fleet_c3_slice_full_length():
+    run_parity(wlm.get_config("c3"), 8, 500, threads=32, check_every=50)
+
+
+def test_small_fleet_c0_full_run():
+    run_parity(wlm.get_config("c0"), 1, 300, threads=32, check_every=25)
+
+
+@pytest.mark.parametrize("kw", [dict(R_max=1), dict(R_max=2), dict(R_max=5), dict(S_greedy=0),
+                                dict(S_greedy=16), dict(S_greedy=1 << 20)])
+def test_small_fleet_window_and_stage_split(kw):
+    run_parity(wlm.get_config("c3", **kw), 4, 260, threads=32, check_every=20)
+
+
+def test_small_fleet_multi_step_and_graph():
+    run_parity(wlm.get_config("c3"), 5, 240, threads=32, launch_steps=8, check_every=1)
+    run_parity(wlm.get_config("c3"), 2, 100, threads=32, graph=True, check_every=10)
+
+
+def test_small_fleet_ragged_and_busy_shapes():
+    # odd worker counts and slot counts, queues that are not a multiple of 128, a hazard high
+    # enough that several requests of a worker end in one step (some at the step they were
+    # admitted), arrival rates that overflow the queue
+    for G, B, W, lam, hz in [(1, 8, 4, 3.0, 0.05), (5, 16, 36, 3.0, 0.05), (7, 40, 100, 6.0, 0.2),
+                             (32, 64, 256, 30.0, 0.3), (31, 56, 252, 12.0, 0.02), (32, 8, 128, 40.0, 0.5)]:
+        cfg = wlm.get_config("c3", G=G, B=B, W=W, init_active=B // 2, init_queue=W // 2, hazard=hz,
+                             arrival=("const", lam), S_greedy=-1)
+        run_parity(cfg, 3, 120, threads=32, check_every=10)
