@@ -55,26 +55,26 @@ def kernel_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(workload: str):
+def recorded_traffic(workload: str, spl: int = 1):
     """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
     profiles/traffic.json, or None if the kernel sources changed since that capture."""
     p = os.path.join(ROOT, "profiles", "traffic.json")
     try:
         rec = json.load(open(p))
         if rec.get("kernel_source_hash") == kernel_source_hash():
-            return rec["bytes_per_launch"].get(workload)
+            return rec["bytes_per_launch"].get(f"{workload}_spl{spl}")
     except Exception:
         pass
     return None
 
 
-def recorded_instructions(workload: str):
+def recorded_instructions(workload: str, spl: int = 1):
     """Warp instructions per launch from the same ncu capture (None if the kernel changed)."""
     p = os.path.join(ROOT, "profiles", "traffic.json")
     try:
         rec = json.load(open(p))
         if rec.get("kernel_source_hash") == kernel_source_hash():
-            return rec.get("warp_instructions_per_launch", {}).get(workload)
+            return rec.get("warp_instructions_per_launch", {}).get(f"{workload}_spl{spl}")
     except Exception:
         pass
     return None
@@ -92,7 +92,7 @@ def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
 
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -104,12 +104,13 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "10"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Summary of the samples taken between host times t0 and t1 (all samples if none fall inside)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is not None:
             self.p.terminate()
@@ -120,6 +121,15 @@ class ClockSampler:
         try:
             self.f.flush()
             rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+            rows = [r for r in rows if len(r) >= 9]
+            if t0 is not None:
+                import datetime
+                def ts(r):
+                    return datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                inside = [r for r in rows if t0 <= ts(r) <= t1]
+                out["samples_total"] = len(rows)
+                if inside:
+                    rows = inside
             sm = [float(r[1]) for r in rows if len(r) >= 9]
             if sm:
                 out["sm_mhz"] = float(np.median(sm))
@@ -221,66 +231,50 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- GPU arm
 class RotatingSets:
-    """R independent instance sets of one configuration, stepped in rotation."""
+    """R independent instance sets of one configuration, stepped in rotation; one call of
+    step() is one launch that advances one set by `spl` decode steps."""
 
-    def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=0, **params):
+    def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=1, spl=1,
+                 **params):
         import torch
         from paper_2605_06113_b200.binding import Router
         self.torch = torch
         self.cfg = wlm.get_config(cfg_name)
-        self.N = n_inst
+        self.N, self.n_sets, self.spl = n_inst, n_sets, spl
         self.sets = []
-        self.router = None
         for r in range(n_sets):
             wl = wlm.make_workload(self.cfg, n_instances=n_inst, first_instance=seed_offset + r * n_inst)
-            if self.router is None:
-                self.wl0 = wl
-                self.router = Router(wl, device=device, threads=threads, **params)
-                arr_rows = [wl.arr_cdf]
-            elif wl.arr_inst_stride:
-                arr_rows.append(wl.arr_cdf)
-            self.sets.append(dict(wl=wl, st=None))
-        # per-instance arrival rows of all sets live in one table; set r starts at row r * N
-        if self.wl0.arr_inst_stride:
-            from paper_2605_06113_b200 import binding
-            import ctypes as C
-            table = np.concatenate(arr_rows, axis=0)
-            self.router.close()
-            big = self.sets[0]["wl"]
-            big_tab = wlm.Workload(cfg=big.cfg, seeds=big.seeds, len_tab=big.len_tab, beta_tab=big.beta_tab,
-                                   arr_cdf=table, arr_period=big.arr_period,
-                                   arr_inst_stride=big.arr_inst_stride, term_cdf=big.term_cdf,
-                                   state=big.state)
-            self.router = Router(big_tab, device=device, threads=threads, **params)
-        # all sets share one allocation per array so that `first_instance` selects the set
-        keys = list(self.sets[0]["wl"].state.keys())
-        cat = {k: np.concatenate([s["wl"].state[k] for s in self.sets], axis=0) for k in keys}
-        self.st = self.router.device_state(cat)
-        self.out = self.router.outputs(n_inst * n_sets)
-        self.out = {k: v[0] for k, v in self.out.items()}      # [R*N, ...]
-        self.out_view = {k: v.unsqueeze(0) for k, v in self.out.items()}
-        self.probs = None
-        if self.cfg.H > 0:
-            ring = max(1, probs_ring)
-            seeds_t = torch.from_numpy(np.concatenate([s["wl"].seeds for s in self.sets]).astype(np.int64)).to(device)
-            tab_t = torch.from_numpy(self.wl0.beta_tab).to(device)
-            self.probs = []
-            for j in range(ring):
-                self.probs.append(wlm.term_probs_torch(self.wl0, j, device, seeds_t=seeds_t, tab_t=tab_t).contiguous())
-        self.n_sets = n_sets
+            router = Router(wl, device=device, threads=threads, **params)
+            st = router.device_state()
+            out = router.outputs(n_inst, n_steps=spl)
+            probs = []
+            if self.cfg.H > 0:
+                seeds_t = torch.from_numpy(wl.seeds.astype(np.int64)).to(device)
+                tab_t = torch.from_numpy(wl.beta_tab).to(device)
+                for j in range(max(1, probs_ring)):
+                    probs.append(torch.stack([wlm.term_probs_torch(wl, j * spl + i, device, seeds_t=seeds_t, tab_t=tab_t)
+                                              for i in range(spl)]).contiguous())
+            calls = [router.prepare(st, out, pr, N=n_inst, first=0, n_steps=spl) for pr in (probs or [None])]
+            self.sets.append(dict(wl=wl, router=router, st=st, out=out, probs=probs, calls=calls))
+        self.router = self.sets[0]["router"]
         self.launch = 0
-        self._calls = {}
 
     def step(self):
-        r = self.launch % self.n_sets
-        j = (self.launch // self.n_sets) % len(self.probs) if self.probs is not None else 0
-        call = self._calls.get((r, j))
-        if call is None:       # argument marshalling is done once per (set, probability buffer)
-            probs = self.probs[j] if self.probs is not None else None
-            call = self.router.prepare(self.st, self.out_view, probs, N=self.N, first=r * self.N)
-            self._calls[(r, j)] = call
-        call()
+        s = self.sets[self.launch % self.n_sets]
+        s["calls"][(self.launch // self.n_sets) % len(s["calls"])]()
         self.launch += 1
+
+    def counters_mean(self):
+        t = self.torch
+        return t.stack([s["out"]["counters"].to(t.float64).mean(dim=(0, 1)) for s in self.sets]).mean(0).cpu().numpy()
+
+    def bad_status(self):
+        return sum(int((s["out"]["status"] & ~1).ne(0).sum().item()) for s in self.sets)
+
+    def close(self):
+        for s in self.sets:
+            s["router"].close()
+        self.sets = []
 
 
 def time_launches(torch, fn, warmup, steps, dist=None):
@@ -358,6 +352,43 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
             "phase_us_at_max_clock": phases}
 
 
+def measure_batched(torch, wname, device, steps, warmup, spl, threads=0, seed_offset=0, dist=None,
+                    sampler=None, probs_ring=2):
+    """Times `steps` decode steps of the batched configuration `wname`, `spl` steps per launch, on
+    enough rotating instance sets that no instance runs past the configuration's length."""
+    cfg = wlm.get_config(wname)
+    N = cfg.N
+    per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
+    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))),
+                 int(np.ceil((steps + warmup) / cfg.steps)))
+    sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
+                        probs_ring=probs_ring, spl=spl)
+    if sampler is not None:
+        sampler.start()
+        time.sleep(0.4)                      # let the sampler come up before the timed region
+    t0 = time.time()
+    ms = time_launches(torch, sets.step, -(-warmup // spl), steps // spl, dist)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
+    cnt = sets.counters_mean()
+    bad = sets.bad_status()
+    tpi = sets.router.params.threads
+    sets.close()
+    del sets
+    torch.cuda.empty_cache()
+    # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
+    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
+    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
+    us_per_launch = 1e3 * ms / (steps // spl)
+    return dict(ms=ms, ms_per_step=ms / steps, us_per_launch=us_per_launch, n_sets=n_sets, N=N,
+                abytes_per_launch=abytes, achieved=abytes / (us_per_launch * 1e-6) / 1e9, bad=bad,
+                clocks=clocks, threads=tpi, launches=steps // spl)
+
+
+def kernel_name(wname):
+    return "br_small_kernel<2,4>" if wname == "c3" else "br_step_kernel<true,8,2,1>"
+
+
 def run_ours(args):
     import torch
     world, rank, local, dist = dist_setup(args)
@@ -365,56 +396,56 @@ def run_ours(args):
     torch.cuda.set_device(local)
     peak, peak_kind = measured_peaks()
 
-    # ---------------- headline: c3 batched ----------------
+    # ---------------- headline: batched, several decode steps per launch ----------------
     wname = args.workload
     cfg = wlm.get_config(wname)
-    N = cfg.N
-    per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
-    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state)))) if wname == "c3" else 2
-    first, _ = shard_of(rank, world, N, n_sets)
-    sets = RotatingSets(wname, N, n_sets, device, seed_offset=first, threads=args.threads, probs_ring=4)
-    sampler = ClockSampler(local)
-    sampler.start()
-    ms = time_launches(torch, sets.step, args.warmup, args.steps, dist)
-    clocks = sampler.stop()
-    cnt = sets.out["counters"].to(torch.float64).view(n_sets, N, 4).mean(dim=(0, 1)).cpu().numpy()
-    bad = int((sets.out["status"] & ~1).ne(0).sum().item())
-    value = world * N * args.steps / (ms * 1e-3)
-    # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
-    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
-    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N
-    achieved = abytes / (ms * 1e-3 / args.steps) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "peak_kind": peak_kind, "traffic": recorded_traffic(wname),
-                "algorithmic_bytes_per_launch": abytes,
-                "kernel": "br_step_kernel<false,0,1,2>" if wname == "c3" else "br_step_kernel<true,8,2,1>"}
-
-    winst = recorded_instructions(wname)
+    spl = args.steps_per_launch if args.steps % args.steps_per_launch == 0 else 1
+    first, _ = shard_of(rank, world, cfg.N, 64)
+    m = measure_batched(torch, wname, device, args.steps, args.warmup, spl, threads=args.threads,
+                        seed_offset=first, dist=dist, sampler=ClockSampler(local))
+    N = m["N"]
+    value = world * N * args.steps / (m["ms"] * 1e-3)
+    roofline = {"bound": "hbm", "achieved": m["achieved"], "peak": peak, "unit": "GB/s",
+                "frac": m["achieved"] / peak, "frac_of_nominal_8TBs": m["achieved"] / NOMINAL_HBM_GBS,
+                "peak_kind": peak_kind, "traffic": recorded_traffic(wname, spl),
+                "algorithmic_bytes_per_launch": m["abytes_per_launch"],
+                "us_per_launch": m["us_per_launch"], "kernel": kernel_name(wname)}
+    winst = recorded_instructions(wname, spl)
+    clocks = m["clocks"]
     if winst:
         # what actually binds the step: instruction issue.  Peak = 148 SMs x 4 schedulers x 1 warp
         # instruction per clock at the SM clock sampled during the run.
         clk = (clocks.get("sm_mhz") or 1965.0) * 1e6
         peak_issue = 148 * 4 * clk
-        ach = winst / (ms * 1e-3 / args.steps)
+        ach = winst / (m["us_per_launch"] * 1e-6)
         roofline["issue"] = {"bound": "alu", "achieved": ach / 1e9, "peak": peak_issue / 1e9,
                              "unit": "G warp-instructions/s", "frac": ach / peak_issue,
                              "warp_instructions_per_launch": winst}
     line = {
         "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
         "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
         "config": {"workload": ("c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.." if wname == "c3"
                                 else "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000.."),
-                   "instances_per_launch": N, "rotating_sets": n_sets,
-                   "l2": f"{n_sets} instance sets stepped in rotation: data touched between two visits "
-                         f"of a set exceeds the 126 MB L2", "threads_per_instance": sets.router.params.threads},
-        "roofline": roofline, "clocks": clocks, "gpu_launches": args.steps,
-        "bad_status_instances": bad,
+                   "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
+                   "l2": f"{m['n_sets']} instance sets stepped in rotation ({spl} decode steps per launch and "
+                         f"set): data touched between two visits of a set exceeds the 126 MB L2; no instance "
+                         f"runs past the configuration's {cfg.steps} steps",
+                   "threads_per_instance": m["threads"]},
+        "roofline": roofline, "clocks": clocks, "gpu_launches": m["launches"],
+        "bad_status_instances": m["bad"],
     }
 
     if rank == 0 and world == 1 and not args.quick and wname == "c3":
+        # the same workload with one decode step per launch (the form the latency path replays)
+        m1 = measure_batched(torch, wname, device, 1920, 80, 1, threads=args.threads)
+        line["single_step_launches"] = {
+            "value": N * 1920 / (m1["ms"] * 1e-3), "unit": UNIT, "ms_per_step": m1["ms_per_step"],
+            "roofline": {"bound": "hbm", "achieved": m1["achieved"], "peak": peak, "unit": "GB/s",
+                         "frac": m1["achieved"] / peak, "traffic": recorded_traffic(wname, 1),
+                         "algorithmic_bytes_per_launch": m1["abytes_per_launch"]},
+            "gpu_launches": 1920}
         # ---------------- end to end through the host-buffer entry point ----------------
         line["e2e"] = e2e_host(torch, device, args)
         # ---------------- extras: c4 batched BR-H, latency path ----------------
@@ -461,19 +492,16 @@ def e2e_host(torch, device, args):
 
 def extras(torch, device, args, peak):
     ex = {}
-    # c4: BR-H batched, term_probs ring of 8 step buffers (1 GiB) and 2 instance sets
-    cfg = wlm.get_config("c4")
-    sets = RotatingSets("c4", cfg.N, 2, device, seed_offset=0, probs_ring=4)
-    ms = time_launches(torch, sets.step, 20, 200)
-    cnt = sets.out["counters"].to(torch.float64).view(2, cfg.N, 4).mean(dim=(0, 1)).cpu().numpy()
-    abytes = algorithmic_bytes(cfg, float(2 * cnt[1] + 20), 1.0 / cfg.delta_T) * cfg.N
-    ach = abytes / (ms * 1e-3 / 200) / 1e9
-    ex["c4_batched"] = {"value": cfg.N * 200 / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms / 200,
-                        "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                                     "frac": ach / peak, "traffic": recorded_traffic("c4"),
-                                     "algorithmic_bytes_per_launch": abytes}}
-    del sets
-    torch.cuda.empty_cache()
+    # c4: BR-H batched (H = 8), 4 decode steps per launch and one step per launch
+    for spl in (4, 1):
+        m = measure_batched(torch, "c4", device, 400, 40, spl)
+        ex["c4_batched" if spl == 4 else "c4_single_step_launches"] = {
+            "value": m["N"] * 400 / (m["ms"] * 1e-3), "unit": UNIT, "ms_per_step": m["ms_per_step"],
+            "steps_per_launch": spl,
+            "roofline": {"bound": "hbm", "achieved": m["achieved"], "peak": peak, "unit": "GB/s",
+                         "frac": m["achieved"] / peak, "traffic": recorded_traffic("c4", spl),
+                         "algorithmic_bytes_per_launch": m["abytes_per_launch"],
+                         "kernel": kernel_name("c4")}}
     # c3 with 16 steps per launch (persistent multi-step form of the same kernel)
     ex["latency"] = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
                      latency_path(torch, "c4", device, 1000)]
@@ -483,8 +511,10 @@ def extras(torch, device, args, peak):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1920)
-    ap.add_argument("--warmup", type=int, default=80)
+    ap.add_argument("--steps", type=int, default=3840)
+    ap.add_argument("--warmup", type=int, default=160)
+    ap.add_argument("--steps-per-launch", type=int, default=8,
+                    help="decode steps advanced by one launch (one br_step call with n_steps); used when it divides --steps")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="headline measurement only")

@@ -74,3 +74,35 @@ def test_c3_full_batch_sampled_instances():
 
 def test_c4_full_batch_sampled_instances():
     _run("c4", 40, 10, 6)
+
+
+def test_c3_full_batch_eight_steps_per_launch():
+    """The launch the benchmark times: 4,096 instances, eight decode steps per launch.  Sampled
+    instances are compared with the checker at every step of every launch."""
+    cfg = wlm.get_config("c3")
+    N, S = cfg.N, 8
+    wl = wlm.make_workload(cfg)
+    r = Router(wl, device="cuda:0")
+    st = r.device_state()
+    out = r.outputs(N, n_steps=S)
+    rng = np.random.default_rng(11)
+    idx = sorted(set([0, N - 1] + [int(x) for x in rng.integers(0, N, 10)]))
+    orcs = {i: oracle.instance_from_workload(wl, i) for i in idx}
+    call = r.prepare(st, out, None, N=N, first=0, n_steps=S)
+    for launch in range(30):
+        call()
+        torch.cuda.synchronize()
+        assert int((out["status"] & ~1).ne(0).sum()) == 0
+        tr = out["trace"]; load = out["load"]
+        assert torch.equal(tr[:, :, 0], load.max(2).values) and torch.equal(tr[:, :, 2], load.sum(2))
+        ah = out["assign"][:, idx].cpu().numpy(); lh = load[:, idx].cpu().numpy(); th = tr[:, idx].cpu().numpy()
+        for j in range(S):
+            for c, i in enumerate(idx):
+                ao, lo, to, _ = orcs[i].step()
+                assert np.array_equal(ah[j, c], ao), (i, launch, j)
+                assert np.array_equal(lh[j, c], lo), (i, launch, j)
+                assert np.array_equal(th[j, c], to), (i, launch, j)
+    fin = state_to_numpy(st)
+    for i in idx:
+        compare_state(cfg, fin, orcs[i], i, 30 * S)
+    r.close()
