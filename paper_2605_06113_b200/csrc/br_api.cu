@@ -108,9 +108,11 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
         // BR-0 on a small fleet: the one-warp-per-instance kernel
         int wpb = ctx->inst_per_block;
         if (wpb > b->n_instances) wpb = b->n_instances;
-        const int nt4 = ctx->p.W <= 128 ? 1 : 2;
-        step_kernel_t kern = nt4 == 1 ? (ctx->p.R_max <= 4 ? br::br_small_kernel<1, 4> : br::br_small_kernel<1, 5>)
-                                      : (ctx->p.R_max <= 4 ? br::br_small_kernel<2, 4> : br::br_small_kernel<2, 5>);
+        const int nt4 = ctx->p.W <= 128 ? 1 : (ctx->p.W <= 256 ? 2 : 4);
+        const bool r4 = ctx->p.R_max <= 4;
+        step_kernel_t kern = nt4 == 1 ? (r4 ? br::br_small_kernel<1, 4> : br::br_small_kernel<1, 5>)
+                           : nt4 == 2 ? (r4 ? br::br_small_kernel<2, 4> : br::br_small_kernel<2, 5>)
+                                      : (r4 ? br::br_small_kernel<4, 4> : br::br_small_kernel<4, 5>);
         a.tpi = 32;
         const int blocks = (b->n_instances + wpb - 1) / wpb;
         kern<<<blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * sizeof(int), stream>>>(a);
@@ -241,9 +243,9 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G;
     }
     ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
-    // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 256 waiting requests,
+    // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 512 waiting requests,
     // arrivals served by one Philox call, and negative queue keys scoring below every waiting request
-    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 256 && p.term_mode != 2 &&
+    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode != 2 &&
                     p.burst_every == 0 && (!p.arr_cdf || p.arr_len <= 64) &&
                     (long long)(G - 1) * p.s_max + 65536 < (1ll << (31 - wl));
     *out = ctx;

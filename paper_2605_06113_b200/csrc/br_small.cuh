@@ -1,7 +1,7 @@
 // BR-0 routing step for small fleets: one warp per instance, no block barrier.
 //
 // Shapes: G <= 32 workers (lane g owns worker g: free slots, load L_g, occupancy word),
-// B <= 64 slots per worker, W <= 256 waiting requests, Eq. 1 scores in 32-bit integers,
+// B <= 64 slots per worker, W <= 512 waiting requests, Eq. 1 scores in 32-bit integers,
 // constant-hazard (or no) terminations, no optional outputs.  Everything else runs on
 // br_step_kernel.
 //
@@ -26,7 +26,7 @@ namespace br {
 constexpr int kSmallBeyond = (int)0x8000FFFFu;   // key of a position beyond the queue (no slot index reaches 0xFFFF)
 
 template <int NT4 /* 128-position groups: W <= 128 * NT4 */, int RM /* window entries kept */>
-__global__ void __maxnreg__(72) br_small_kernel(const StepArgs a)
+__global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpb = blockDim.x >> 5;
