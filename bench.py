@@ -349,17 +349,20 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
             "host_p50_us": float(np.percentile(h, 50)), "host_p95_us": float(np.percentile(h, 95)),
             "host_p99_us": float(np.percentile(h, 99)), "device_p50_us": float(np.percentile(d, 50)),
             "device_p99_us": float(np.percentile(d, 99)),
-            "phase_us_at_max_clock": phases}
+            "phase_us_at_max_clock": phases,
+            "phase_note": "phase split taken with the kernel's cycle counters on br_step_kernel (the "
+                          "kernel that offers them); the latencies above are those of the kernel the "
+                          "library picks for the shape"}
 
 
 def measure_batched(torch, wname, device, steps, warmup, spl, threads=0, seed_offset=0, dist=None,
-                    sampler=None, probs_ring=2):
+                    sampler=None, probs_ring=2, min_sets=0):
     """Times `steps` decode steps of the batched configuration `wname`, `spl` steps per launch, on
     enough rotating instance sets that no instance runs past the configuration's length."""
     cfg = wlm.get_config(wname)
     N = cfg.N
     per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
-    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))),
+    n_sets = max(2, min_sets, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))),
                  int(np.ceil((steps + warmup) / cfg.steps)))
     sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
                         probs_ring=probs_ring, spl=spl)
@@ -502,7 +505,7 @@ def extras(torch, device, args, peak):
                          "frac": m["achieved"] / peak, "traffic": recorded_traffic("c4", spl),
                          "algorithmic_bytes_per_launch": m["abytes_per_launch"],
                          "kernel": kernel_name("c4")}}
-    # c3 with 16 steps per launch (persistent multi-step form of the same kernel)
+    # latency path: one instance, one graph-replayed step per decode step
     ex["latency"] = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
                      latency_path(torch, "c4", device, 1000)]
     return ex
