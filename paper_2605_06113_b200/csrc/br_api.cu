@@ -239,8 +239,23 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         }
         volatile double aD = p.alpha * D;
         a.aD = aD; a.beta = p.beta;
+        // The single-request arg-max may use the concavity of Eq. 2 only if no segment slope
+        // alpha D - beta sum_{h in P} d_h (P any set of passed kinks) is within rounding distance of
+        // zero: then fp64 scores of integer lengths are strictly ordered on both sides of the peak.
+        {
+            const int n = H + 1;
+            double min_abs = 1e300;
+            for (unsigned mask = 0; mask < (1u << n); ++mask) {
+                double w = 0.0;
+                for (int h = 0; h < n; ++h) if (mask >> h & 1u) w += a.d[h];
+                const double sl = fabs(a.aD - p.beta * w);
+                if (sl < min_abs) min_abs = sl;
+            }
+            const double err = 4.0 * (H + 5) * 1.1102230246251565e-16 * (a.aD + p.beta * D) * (double)p.s_max;
+            a.peak_ok = (min_abs > err && min_abs > 1e-9) ? 1 : 0;
+        }
     } else {
-        a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G;
+        a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G; a.peak_ok = 0;
     }
     ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
     // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 512 waiting requests,

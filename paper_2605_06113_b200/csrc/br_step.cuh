@@ -34,6 +34,7 @@ struct StepArgs {
     int32_t len_shift;
     int32_t burst_every, burst_size;
     double aD, beta;
+    int32_t peak_ok;            // Eq. 2: every slope alpha D - beta sum_{h in P} d_h is clearly off zero (br_create)
     double d[BR_MAX_H + 1];
     int32_t N, first_instance, n_steps;
     int32_t tpi, smem_per_inst;  // threads and shared-memory bytes per instance
@@ -558,6 +559,42 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int src = warp_argmax_lane32(bk, (unsigned)bkey & posmask, wk);
                     const int res = __shfl_sync(kFull, bkey, src);
                     return res > 0 ? res : 0;
+                } else if (a.peak_ok) {
+                    // Eq. 2 is concave and piecewise linear in s with kinks at the m_{g,h}: it rises up
+                    // to s* = the smallest kink at which the slope alpha D - beta sum_{m_h <= kink} d_h
+                    // is no longer positive, and falls after it.  br_create has checked that no such
+                    // slope is within rounding distance of zero, so the fp64 scores of integer lengths
+                    // are strictly ordered on either side, and the arg-max is the largest s <= s* or the
+                    // smallest s > s* (earliest arrival among equal lengths): two integer scans and two
+                    // evaluations of Eq. 2.
+                    double mine = 0.0;
+#pragma unroll
+                    for (int h = 0; h <= HM; ++h) if (lane == h) mine = sc.md[h];
+                    double wsum = 0.0;
+#pragma unroll
+                    for (int h = 0; h <= HM; ++h) if (h <= H && sc.md[h] <= mine) wsum = __dadd_rn(wsum, a.d[h]);
+                    const bool past = lane <= H && !(a.aD > __dmul_rn(a.beta, wsum));
+                    const int sstar = (int)__reduce_min_sync(kFull, past ? (unsigned)(int)mine : 0x7FFFFFFFu);
+                    const int thr = sstar >= (1 << (31 - WL)) ? 0x7FFFFFFF : ((sstar << WL) | (int)posmask);
+                    int below = 0; unsigned above = 0x7FFFFFFFu;
+#pragma unroll 4
+                    for (int t = 0; t < n_tiles; ++t) {
+                        const int idx = (t << 5) + lane;
+                        const int qk = idx < n_w ? q_key[idx] : 0;
+                        if (qk > 0) {
+                            if (qk <= thr) below = max(below, qk);
+                            else above = min(above, (unsigned)qk ^ posmask);
+                        }
+                    }
+                    const int ka = __reduce_max_sync(kFull, below);
+                    const unsigned ab = __reduce_min_sync(kFull, above);
+                    const int kb = ab == 0x7FFFFFFFu ? 0 : (int)(ab ^ posmask);
+                    const long long fa = ka > 0 ? sc.key(a, ka >> WL) : kNoKey;
+                    const long long fb = kb > 0 ? sc.key(a, kb >> WL) : kNoKey;
+                    if (fa > fb) return ka;
+                    if (fb > fa) return kb;
+                    if (ka <= 0) return 0;
+                    return ((unsigned)ka & posmask) > ((unsigned)kb & posmask) ? ka : kb;
                 } else {
                     // Horizon-safe requests (s <= min_h m_{g,h}) score alpha D s exactly, which grows
                     // with s: of those only the largest key per lane is scored; the others in full.

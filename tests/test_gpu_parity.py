@@ -127,3 +127,11 @@ def test_small_fleet_ragged_and_busy_shapes():
         cfg = wlm.get_config("c3", G=G, B=B, W=W, init_active=B // 2, init_queue=W // 2, hazard=hz,
                              arrival=("const", lam), S_greedy=-1)
         run_parity(cfg, 3, 120, threads=32, check_every=10)
+
+
+def test_brh_flat_slope_takes_the_full_scan():
+    # alpha D = beta (d_0 + d_1): one segment of Eq. 2 is flat, scores tie across lengths, and the
+    # single-request arg-max must scan every request (earliest arrival among equal scores)
+    run_parity(wlm.get_config("c2", H=1, alpha=1.0, beta=1.0, gamma=1.0, gate=0.0, delta_T=1), 2, 150,
+               check_every=25)
+    run_parity(wlm.get_config("c4", H=2, alpha=1.0, beta=1.0, gamma=1.0), 1, 60, check_every=20)

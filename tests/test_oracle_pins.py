@@ -634,3 +634,50 @@ def test_best_subset_agrees_with_reachable_sums_and_two_probe_rule():
         H = int(rng.integers(1, 5)); mh = rng.integers(0, 900, H + 1)
         mask, f = oracle.best_subset(1, G, H, 1.0, 4.0, 0.5, mh, win, lim)
         assert f == max(oracle.f_brh(H, 1.0, 4.0, 0.5, d, mh) for d in sums)
+
+
+def test_eq2_single_request_argmax_sits_next_to_the_peak():
+    """Eq. 2 is concave and piecewise linear in Delta with kinks at the margins m_{g,h}: it rises
+    until the slope alpha D - beta sum_{m_h <= Delta} gamma^h turns non-positive and falls after.
+    With every such slope well away from zero, the fp64 values at integer lengths are strictly
+    ordered on either side of that kink s*, so the best single request is the largest s <= s* or
+    the smallest s > s*.  (The CUDA path relies on this for its single-request arg-max.)"""
+    rng = np.random.default_rng(53)
+    for alpha, beta, gamma in [(1.0, 14.67, 0.64), (1.0, 43.0, 0.86), (1.0, 48.0, 0.9), (2.0, 3.0, 0.5)]:
+        for _ in range(60):
+            H = int(rng.integers(1, 9))
+            m = np.sort(rng.integers(0, 5000, H + 1))[rng.permutation(H + 1)]
+            d, D = oracle.discount(H, gamma)
+            # the statement needs every segment slope clearly off zero (the library checks the same
+            # at br_create and otherwise scans every request): e.g. (2, 3, 0.5) has a flat segment at H = 1
+            slopes = [alpha * D - beta * sum(d[h] for h in range(H + 1) if mask >> h & 1)
+                      for mask in range(1 << (H + 1))]
+            if min(abs(x) for x in slopes) < 1e-9:
+                continue
+            # s*: smallest kink whose passed weight makes the slope non-positive
+            order = np.argsort(m, kind="stable")
+            sstar = None
+            for i in order:
+                w = d[m <= m[i]].sum()
+                if alpha * D - beta * w <= 0:
+                    sstar = int(m[i]); break
+            sizes = [int(x) for x in rng.integers(1, 9000, 40)]
+            f = [oracle.f_brh(H, alpha, beta, gamma, s, m) for s in sizes]
+            best = max(range(len(sizes)), key=lambda i: (f[i], -i))           # earliest on ties
+            below = [i for i in range(len(sizes)) if sstar is None or sizes[i] <= sstar]
+            above = [i for i in range(len(sizes)) if sstar is not None and sizes[i] > sstar]
+            cand = []
+            if below:
+                top = max(sizes[i] for i in below); cand.append(min(i for i in below if sizes[i] == top))
+            if above:
+                low = min(sizes[i] for i in above); cand.append(min(i for i in above if sizes[i] == low))
+            pick = max(cand, key=lambda i: (f[i], -i))
+            assert pick == best
+            # strict order of the fp64 values on either side of the peak
+            grid = sorted(set(sizes))
+            vals = [oracle.f_brh(H, alpha, beta, gamma, s, m) for s in grid]
+            for a_, b_, fa, fb in zip(grid, grid[1:], vals, vals[1:]):
+                if sstar is None or b_ <= sstar:
+                    assert fb > fa
+                elif a_ >= sstar:
+                    assert fb < fa
