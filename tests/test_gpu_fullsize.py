@@ -106,3 +106,41 @@ def test_c3_full_batch_eight_steps_per_launch():
     for i in idx:
         compare_state(cfg, fin, orcs[i], i, 30 * S)
     r.close()
+
+
+def test_c4_full_batch_four_steps_per_launch():
+    """The BR-H launch the benchmark times: 1,024 instances, four decode steps per launch, the
+    classifier output of the four steps passed as one block."""
+    cfg = wlm.get_config("c4")
+    N, S = cfg.N, 4
+    wl = wlm.make_workload(cfg)
+    r = Router(wl, device="cuda:0")
+    st = r.device_state()
+    out = r.outputs(N, n_steps=S)
+    rng = np.random.default_rng(13)
+    idx = sorted(set([0, N - 1] + [int(x) for x in rng.integers(0, N, 4)]))
+    orcs = {i: oracle.instance_from_workload(wl, i) for i in idx}
+    seeds_t = torch.from_numpy(wl.seeds.astype(np.int64)).cuda()
+    tab_t = torch.from_numpy(wl.beta_tab).cuda()
+    probs_t = torch.empty((S, N, cfg.G, cfg.B, cfg.H), dtype=torch.float32, device="cuda:0")
+    call = r.prepare(st, out, probs_t, N=N, first=0, n_steps=S)
+    for launch in range(6):
+        for j in range(S):
+            wlm.term_probs_torch(wl, launch * S + j, "cuda:0", seeds_t=seeds_t, tab_t=tab_t, out=probs_t[j])
+        call()
+        torch.cuda.synchronize()
+        assert int((out["status"] & ~1).ne(0).sum()) == 0
+        tr = out["trace"]; load = out["load"]
+        assert torch.equal(tr[:, :, 0], load.max(2).values) and torch.equal(tr[:, :, 2], load.sum(2))
+        ah = out["assign"][:, idx].cpu().numpy(); lh = load[:, idx].cpu().numpy(); th = tr[:, idx].cpu().numpy()
+        for j in range(S):
+            probs_np = wlm.term_probs_np(wl, launch * S + j, instances=idx)
+            for c, i in enumerate(idx):
+                ao, lo, to, _ = orcs[i].step(probs_np[c])
+                assert np.array_equal(ah[j, c], ao), (i, launch, j)
+                assert np.array_equal(lh[j, c], lo), (i, launch, j)
+                assert np.array_equal(th[j, c], to), (i, launch, j)
+    fin = state_to_numpy(st)
+    for i in idx:
+        compare_state(cfg, fin, orcs[i], i, 6 * S)
+    r.close()
