@@ -115,7 +115,7 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
                                       : (r4 ? br::br_small_kernel<4, 4> : br::br_small_kernel<4, 5>);
         a.tpi = 32;
         const int blocks = (b->n_instances + wpb - 1) / wpb;
-        kern<<<blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * sizeof(int), stream>>>(a);
+        kern<<<blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * 2 * sizeof(int), stream>>>(a);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
         return BR_OK;

@@ -6,8 +6,8 @@
 // br_step_kernel.
 //
 // A lane owns the queue positions (t * 32 + lane) * 4 + j, j < 4: prompt lengths, ids and
-// assignments move as 16-byte vectors, and within a lane positions ascend.  The queue lives in
-// shared memory as packed keys (s << wl | inverted position) so that "largest s, earliest
+// assignments move as 16-byte vectors, and within a lane positions ascend.  For the length of a
+// launch the queue lives in shared memory (ids beside it) as packed keys (s << wl | inverted position) so that "largest s, earliest
 // arrival" is one integer max; an admitted entry becomes 0x80000000 | slot and a position
 // beyond the queue 0x8000FFFF.  Both are negative: they lose every max of keys, and read as
 // a prompt length they score below any waiting request (range checked on the host), so the
@@ -33,7 +33,8 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
     const int row = blockIdx.x * wpb + wib;
     if (row >= a.N) return;
     const int inst = a.first_instance + row;
-    int *q_key = reinterpret_cast<int *>(smem_all) + wib * (NT4 * 128);
+    int *q_key = reinterpret_cast<int *>(smem_all) + wib * (2 * NT4 * 128);          // [NT4 * 128] packed keys
+    unsigned *q_id = reinterpret_cast<unsigned *>(q_key + NT4 * 128);                 // [NT4 * 128] request ids
 
     const int G = a.G, B = a.B, W = a.W, WL = a.wl, A = G * B;
     const unsigned posmask = (1u << WL) - 1u;
@@ -64,22 +65,33 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
         occ = a.ws.occ[(size_t)inst * G + lane] | ~slots;
     }
 
+    // ---- the queue moves to shared memory once per launch: packed keys and ids ----
+#pragma unroll
+    for (int t = 0; t < NT4; ++t) {
+        const int p0 = (t * 32 + lane) * 4;
+        int4 sv = make_int4(0, 0, 0, 0); uint4 iv = make_uint4(0u, 0u, 0u, 0u);
+        if (p0 < W) {
+            sv = *reinterpret_cast<const int4 *>(g_qs + p0);
+            iv = *reinterpret_cast<const uint4 *>(g_qid + p0);
+        }
+        int4 kk;
+        kk.x = p0 + 0 < n_w ? (sv.x << WL) | (int)(posmask - (unsigned)(p0 + 0)) : kSmallBeyond;
+        kk.y = p0 + 1 < n_w ? (sv.y << WL) | (int)(posmask - (unsigned)(p0 + 1)) : kSmallBeyond;
+        kk.z = p0 + 2 < n_w ? (sv.z << WL) | (int)(posmask - (unsigned)(p0 + 2)) : kSmallBeyond;
+        kk.w = p0 + 3 < n_w ? (sv.w << WL) | (int)(posmask - (unsigned)(p0 + 3)) : kSmallBeyond;
+        *reinterpret_cast<int4 *>(q_key + p0) = kk;
+        *reinterpret_cast<uint4 *>(q_id + p0) = iv;
+    }
+    __syncwarp();
+
 #pragma unroll 1
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + row;
         int32_t *assign = a.assign_out + orow * W;
-
-        // ---- queue rows: prompt lengths and ids of this lane's positions ----
-        int4 sv[NT4]; uint4 iv[NT4];
 #pragma unroll
         for (int t = 0; t < NT4; ++t) {
             const int p0 = (t * 32 + lane) * 4;
-            sv[t] = make_int4(0, 0, 0, 0); iv[t] = make_uint4(0u, 0u, 0u, 0u);
-            if (p0 < W) {
-                sv[t] = *reinterpret_cast<const int4 *>(g_qs + p0);
-                iv[t] = *reinterpret_cast<const uint4 *>(g_qid + p0);
-                *reinterpret_cast<int4 *>(assign + p0) = make_int4(-1, -1, -1, -1);
-            }
+            if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(-1, -1, -1, -1);
         }
 
         // ================= ARRIVE (Section 2.2) =================
@@ -108,18 +120,6 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
         int pend = 0;
         if (pj >= 0) pend = g_base[lane * B + pj];
 
-        // packed keys of the queue as it was
-#pragma unroll
-        for (int t = 0; t < NT4; ++t) {
-            const int p0 = (t * 32 + lane) * 4;
-            int4 kk;
-            kk.x = p0 + 0 < n_w ? (sv[t].x << WL) | (int)(posmask - (unsigned)(p0 + 0)) : kSmallBeyond;
-            kk.y = p0 + 1 < n_w ? (sv[t].y << WL) | (int)(posmask - (unsigned)(p0 + 1)) : kSmallBeyond;
-            kk.z = p0 + 2 < n_w ? (sv[t].z << WL) | (int)(posmask - (unsigned)(p0 + 2)) : kSmallBeyond;
-            kk.w = p0 + 3 < n_w ? (sv[t].w << WL) | (int)(posmask - (unsigned)(p0 + 3)) : kSmallBeyond;
-            *reinterpret_cast<int4 *>(q_key + p0) = kk;
-        }
-        __syncwarp();
         const int n_w_old = n_w;
         const uint32_t id0 = next_id;
         int n_take = W - n_w;
@@ -136,6 +136,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
                 const int s = a.len_tab[w >> a.len_shift];
                 const int pos = n_w_old + j;
                 q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
+                q_id[pos] = id0 + (unsigned)j;
             }
         }
         n_w += n_take;
@@ -287,33 +288,38 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
             }
         }
 
-        // ============ stable queue compaction; ids of the admitted requests ============
+        // ============ stable queue compaction in shared memory; ids of the admitted requests ============
+        // An entry that moves down by d positions keeps its length and gains d in the inverted
+        // position field: its key grows by d.
         {
             int run = 0;                                  // entries kept in the groups before this one
 #pragma unroll
             for (int t = 0; t < NT4; ++t) {
                 const int p0 = (t * 32 + lane) * 4;
                 if (t * 128 >= n_w) break;
-                if (t * 128 + 128 <= first_rm && t * 128 + 128 <= n_w_old) { run += 128; continue; }   // nothing moves here
+                if (t * 128 + 128 <= first_rm) { run += 128; continue; }     // nothing before the first admission moves
                 const int4 kk = *reinterpret_cast<const int4 *>(q_key + p0);
+                const uint4 ii = *reinterpret_cast<const uint4 *>(q_id + p0);
                 const int ke[4] = {kk.x, kk.y, kk.z, kk.w};
-                const unsigned idv[4] = {iv[t].x, iv[t].y, iv[t].z, iv[t].w};
+                const unsigned idv[4] = {ii.x, ii.y, ii.z, ii.w};
                 int below = run;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) below += __popc(__ballot_sync(kFull, ke[j] > 0) & lt);
+                __syncwarp();                             // the group is read before any of it is overwritten
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int pos = p0 + j;
-                    const unsigned id = pos < n_w_old ? idv[j] : id0 + (unsigned)(pos - n_w_old);
                     if (ke[j] > 0) {
-                        if (below != pos || pos >= n_w_old) { g_qs[below] = ke[j] >> WL; g_qid[below] = id; }
+                        if (below != pos) { q_key[below] = ke[j] + (pos - below); q_id[below] = idv[j]; }
                         ++below;
                     } else if (g_aid && ke[j] != kSmallBeyond) {
-                        g_aid[ke[j] & 0x7FFFFFFF] = id;
+                        g_aid[ke[j] & 0x7FFFFFFF] = idv[j];
                     }
                 }
                 run = __shfl_sync(kFull, below, 31);
             }
+            for (int j = n_left + lane; j < n_w; j += 32) q_key[j] = kSmallBeyond;   // vacated tail
+            __syncwarp();
         }
         n_w = n_left;
 
@@ -342,6 +348,18 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
     }
 
     // ---- snapshot write-back ----
+#pragma unroll
+    for (int t = 0; t < NT4; ++t) {
+        const int p0 = (t * 32 + lane) * 4;
+        if (p0 < W) {
+            const int4 kk = *reinterpret_cast<const int4 *>(q_key + p0);
+            int4 sv;
+            sv.x = kk.x > 0 ? kk.x >> WL : 0; sv.y = kk.y > 0 ? kk.y >> WL : 0;
+            sv.z = kk.z > 0 ? kk.z >> WL : 0; sv.w = kk.w > 0 ? kk.w >> WL : 0;
+            *reinterpret_cast<int4 *>(g_qs + p0) = sv;
+            *reinterpret_cast<uint4 *>(g_qid + p0) = *reinterpret_cast<const uint4 *>(q_id + p0);
+        }
+    }
     if (lane < G) {
         a.ws.load[(size_t)inst * G + lane] = (long long)L;
         a.ws.nact[(size_t)inst * G + lane] = B - cap;
