@@ -89,9 +89,31 @@ int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_work
     return BR_OK;
 }
 
+// Launch with programmatic stream serialisation: the blocks of this launch may become resident
+// while the previous kernel of the stream is still draining.  Both step kernels open with
+// griddepcontrol.wait, which returns only when every earlier kernel of the stream has completed
+// and its writes are visible, so only launch latency and block scheduling overlap.
+cudaError_t launch_overlapped(step_kernel_t kern, int blocks, int threads, size_t smem, cudaStream_t stream,
+                              const StepArgs &a, bool overlap)
+{
+    if (!overlap) {                      // plain launch (stream capture)
+        kern<<<blocks, threads, smem, stream>>>(a);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)blocks); cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
 int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *ws,
                 const br_waiting_queue *wq, const float *term_probs, int32_t *assign_out,
-                const br_load_out *out, cudaStream_t stream)
+                const br_load_out *out, cudaStream_t stream, bool overlap = true)
 {
     StepArgs a = ctx->base;
     a.N = b->n_instances;
@@ -115,8 +137,8 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
                                       : (r4 ? br::br_small_kernel<4, 4> : br::br_small_kernel<4, 5>);
         a.tpi = 32;
         const int blocks = (b->n_instances + wpb - 1) / wpb;
-        kern<<<blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * 2 * sizeof(int), stream>>>(a);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_overlapped(kern, blocks, 32 * wpb, (size_t)wpb * nt4 * 128 * 2 * sizeof(int), stream, a, overlap);
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
         return BR_OK;
     }
@@ -134,8 +156,8 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.block_sync = (per_block > 1 && b->n_instances % per_block == 0) ? 1 : 0;
     a.smem_per_inst = (int32_t)ctx->smem;
     const int blocks = (b->n_instances + per_block - 1) / per_block;
-    kern<<<blocks, tpi * per_block, ctx->smem * per_block, stream>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_overlapped(kern, blocks, tpi * per_block, ctx->smem * per_block, stream, a, overlap);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
     return BR_OK;
 }
@@ -289,7 +311,7 @@ int br_graph_capture(br_ctx *ctx, const br_instance_batch *batch, br_worker_stat
     BR_CUDA(cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking));
     cudaError_t e = cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) { cudaStreamDestroy(cap); return cuda_fail(e, "cudaStreamBeginCapture"); }
-    rc = launch_step(ctx, batch, ws, wq, term_probs, assign_out, out, cap);
+    rc = launch_step(ctx, batch, ws, wq, term_probs, assign_out, out, cap, false);
     e = cudaStreamEndCapture(cap, &ctx->graph);
     cudaStreamDestroy(cap);
     if (rc != BR_OK) return rc;

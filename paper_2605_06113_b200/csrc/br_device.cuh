@@ -13,6 +13,15 @@ constexpr int kNoIdx = 0x7FFFFFFF;
 
 enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2 };
 
+// First statements of a step kernel: let the next kernel of the stream start becoming resident,
+// then wait until every earlier kernel of the stream has completed and flushed its writes
+// (both are no-ops for a launch without programmatic stream serialisation).
+__device__ __forceinline__ void stream_order_gate()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0, k1).
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
                                                uint32_t k0, uint32_t k1)

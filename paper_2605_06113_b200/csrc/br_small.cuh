@@ -31,6 +31,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
     extern __shared__ __align__(16) unsigned char smem_all[];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const int row = blockIdx.x * wpb + wib;
+    stream_order_gate();
     if (row >= a.N) return;
     const int inst = a.first_instance + row;
     int *q_key = reinterpret_cast<int *>(smem_all) + wib * (2 * NT4 * 128);          // [NT4 * 128] packed keys

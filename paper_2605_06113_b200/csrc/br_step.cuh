@@ -164,6 +164,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     const int NT = a.tpi;
     const int tid = threadIdx.x % NT, lane = tid & 31, warp = tid >> 5;
     const int in_block = threadIdx.x / NT, per_block = blockDim.x / NT;
+    stream_order_gate();
     if (blockIdx.x * per_block + in_block >= a.N) return;            // whole instance groups only
     unsigned char *smem_raw = smem_all + (size_t)in_block * a.smem_per_inst;
     // Instance-wide barrier.  Single-warp instances that share a block may also be aligned with a
