@@ -223,6 +223,20 @@ int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_s
 int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int32_t n_requests,
               const int64_t *Lh, const int32_t *cap, double *F, int32_t *best_g);
 
+/*
+ * The Stage-2 subproblem alone, solved exactly for windows larger than the R_max <= 5 of br_step
+ * (Algorithms 1 and 2, Stage 2; Appendix "Bit-set subset selection": the score depends on Q only
+ * through Delta(Q)).  For each of batch.n_instances problems: win [N][R] holds the prompt lengths
+ * of the window (1 <= R <= 20; bit j of a mask selects entry j), margins [N][H+1] the worker's
+ * m_{g,h} (H = 0: m_g), lim [N] the largest subset size (the worker's free slots).  Writes
+ * best_mask [N] = the non-empty subset with |Q| <= lim and the highest F_g(Q) (Eq. 1 / Eq. 2 as
+ * in br_step), lowest mask on ties, 0 if lim < 1; best_F [N] (may be NULL) its score.  All 2^R - 1
+ * subsets are enumerated, one thread block per problem.  Device pointers; asynchronous on
+ * batch.stream; BR_EINVAL for null pointers or R outside [1, 20].
+ */
+int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *win, int32_t R,
+                   const int64_t *margins, const int32_t *lim, uint32_t *best_mask, double *best_F);
+
 /* Frees the context, its staging buffers and graph.  NULL is accepted. */
 int br_destroy(br_ctx *ctx);
 

@@ -55,7 +55,7 @@ class BrLoadOut(C.Structure):
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
            "br_step_host_static",
-           "br_fscore", "br_destroy", "br_strerror", "br_version"]
+           "br_fscore", "br_best_subset", "br_destroy", "br_strerror", "br_version"]
 
 _lib = None
 
@@ -85,6 +85,8 @@ def lib():
         L.br_step_host_static.argtypes = step_args + [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.br_fscore.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.br_best_subset.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_destroy.argtypes = [C.c_void_p]
         L.br_strerror.restype = C.c_char_p
         L.br_strerror.argtypes = [C.c_int]
@@ -264,6 +266,15 @@ class Router:
                              _ptr(F), _ptr(best_g))
         if rc != BR_OK:
             raise BrError(rc, "br_fscore")
+
+
+    def best_subset(self, win, margins, lim, best_mask, best_F=None, N=None, first=0, stream=None):
+        N = win.shape[0] - first if N is None else N
+        b = BrInstanceBatch(n_instances=N, first_instance=first, n_steps=1, stream=self._stream(stream))
+        rc = lib().br_best_subset(self._h, C.byref(b), _ptr(win), int(win.shape[1]), _ptr(margins), _ptr(lim),
+                                  _ptr(best_mask), _ptr(best_F))
+        if rc != BR_OK:
+            raise BrError(rc, "br_best_subset")
 
 
 def state_to_numpy(st) -> Dict[str, np.ndarray]:

@@ -10,6 +10,7 @@
 #include "br_step.cuh"
 #include "br_small.cuh"
 #include "br_fscore.cuh"
+#include "br_subset.cuh"
 
 using br::StepArgs;
 
@@ -535,6 +536,28 @@ int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int
     br::br_fscore_kernel<<<grid, 256, 0, (cudaStream_t)batch->stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_fscore launch");
+    return BR_OK;
+}
+
+int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *win, int32_t R,
+                   const int64_t *margins, const int32_t *lim, uint32_t *best_mask, double *best_F)
+{
+    if (!ctx || !batch || !win || !margins || !lim || !best_mask) return BR_EINVAL;
+    if (batch->n_instances < 0 || batch->first_instance < 0 || R < 1 || R > br::kSubsetMaxR) return BR_EINVAL;
+    if (misaligned(win, 4) || misaligned(margins, 8) || misaligned(lim, 4) || misaligned(best_mask, 4) ||
+        (best_F && misaligned(best_F, 8)))
+        return BR_EINVAL;
+    if (batch->n_instances == 0) return BR_OK;
+    br::SubsetArgs a;
+    memset(&a, 0, sizeof(a));
+    a.f.G = ctx->G; a.f.H = ctx->H; a.f.fp = ctx->p.score_mode == 1;
+    a.f.aD = ctx->base.aD; a.f.beta = ctx->base.beta;
+    for (int h = 0; h <= BR_MAX_H; ++h) a.f.d[h] = ctx->base.d[h];
+    a.R = R; a.first_instance = batch->first_instance;
+    a.win = win; a.m = margins; a.lim = lim; a.best_mask = best_mask; a.best_F = best_F;
+    br::br_subset_kernel<<<batch->n_instances, 256, 0, (cudaStream_t)batch->stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "br_best_subset launch");
     return BR_OK;
 }
 
