@@ -111,7 +111,7 @@ typedef struct {
 
 typedef struct {
     int32_t n_instances;    /* instances in this call                                           */
-    int32_t first_instance; /* row offset into every per-instance array                         */
+    int32_t first_instance; /* row offset into every per-instance array, state and outputs alike   */
     int32_t n_steps;        /* consecutive decode steps run by this one launch; <= 0 -> 1.  With
                                n_steps > 1, term_probs, assign_out and every br_load_out array
                                hold n_steps consecutive per-step blocks of n_instances rows,
@@ -174,7 +174,9 @@ int br_graph_step(br_ctx *ctx);
  * Host-buffer variant: every array pointer in worker_state, waiting_queue, term_probs,
  * assign_out and load_out is a HOST pointer (pinned memory gives asynchronous copies).
  * Copies the snapshot to device staging owned by ctx (grown on demand with cudaMalloc),
- * runs the step, copies state and results back and synchronises the stream.
+ * runs the step, copies state and results back and synchronises the stream.  Batches of 512
+ * instances or more go through in chunks of instances on three internal streams (created on
+ * first use), so that uploads, kernels and downloads of different chunks overlap.
  * h2d_bytes / d2h_bytes, if not NULL, receive the bytes moved in each direction.
  * batch.n_steps must be 1 and batch.first_instance 0.
  */

@@ -30,6 +30,9 @@ struct br_ctx {
     // host-buffer path
     void *stage;
     size_t stage_bytes;
+    cudaStream_t pipe[3];     // copy-in, kernel and copy-out streams of the chunked host-buffer step
+    cudaEvent_t pipe_ev[2 * 8 + 2];
+    bool pipe_ready;
 };
 
 namespace {
@@ -385,22 +388,65 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         if (e != cudaSuccess) { cuda_fail(e, "cudaMalloc(staging)"); return BR_ENOMEM; }
         ctx->stage_bytes = total;
     }
+    // per-instance row size of every block (all blocks are [N][row] arrays)
     size_t off = 0; int64_t up = 0, down = 0;
     for (Blk &b : blks) {
         if (!b.bytes) continue;
         *b.dev = (char *)ctx->stage + off;
         off += (b.bytes + 255) & ~(size_t)255;
-        if (b.in) { BR_CUDA(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, st)); up += (int64_t)b.bytes; }
+        if (b.in) up += (int64_t)b.bytes;
+        if (b.out) down += (int64_t)b.bytes;
     }
     br_instance_batch db = *batch; db.n_steps = 1;
     int rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
     if (rc != BR_OK) return rc;
-    rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
-    if (rc != BR_OK) return rc;
-    for (Blk &b : blks) {
-        if (!b.bytes || !b.out) continue;
-        BR_CUDA(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, st));
-        down += (int64_t)b.bytes;
+    // Large batches go through in chunks of instances on three streams: the upload of chunk c + 1,
+    // the kernel of chunk c and the download of chunk c - 1 overlap (the two copy directions use
+    // separate engines).  Every chunk is a contiguous range of rows of every array.
+    const int n_chunks = N >= 2048 ? 8 : (N >= 512 ? 4 : 1);
+    if (n_chunks > 1 && !ctx->pipe_ready) {
+        for (int i = 0; i < 3; ++i) BR_CUDA(cudaStreamCreateWithFlags(&ctx->pipe[i], cudaStreamNonBlocking));
+        for (int i = 0; i < 2 * 8 + 2; ++i) BR_CUDA(cudaEventCreateWithFlags(&ctx->pipe_ev[i], cudaEventDisableTiming));
+        ctx->pipe_ready = true;
+    }
+    cudaStream_t s_in = st, s_k = st, s_out = st;
+    if (n_chunks > 1) {
+        s_in = ctx->pipe[0]; s_k = ctx->pipe[1]; s_out = ctx->pipe[2];
+        BR_CUDA(cudaEventRecord(ctx->pipe_ev[16], st));              // everything queued on the caller's stream first
+        BR_CUDA(cudaStreamWaitEvent(s_in, ctx->pipe_ev[16], 0));
+        BR_CUDA(cudaStreamWaitEvent(s_k, ctx->pipe_ev[16], 0));
+        BR_CUDA(cudaStreamWaitEvent(s_out, ctx->pipe_ev[16], 0));
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t i0 = N * (size_t)c / n_chunks, i1 = N * (size_t)(c + 1) / n_chunks;
+        for (Blk &b : blks) {
+            if (!b.bytes || !b.in) continue;
+            const size_t row = b.bytes / N;
+            BR_CUDA(cudaMemcpyAsync((char *)*b.dev + i0 * row, (const char *)b.host + i0 * row, (i1 - i0) * row,
+                                    cudaMemcpyHostToDevice, s_in));
+        }
+        if (n_chunks > 1) {
+            BR_CUDA(cudaEventRecord(ctx->pipe_ev[c], s_in));
+            BR_CUDA(cudaStreamWaitEvent(s_k, ctx->pipe_ev[c], 0));
+        }
+        br_instance_batch cb = db;
+        cb.first_instance = (int32_t)i0; cb.n_instances = (int32_t)(i1 - i0);
+        rc = launch_step(ctx, &cb, &dws, &dwq, d_probs, d_assign, &dout, s_k);   // rows are addressed through first_instance
+        if (rc != BR_OK) return rc;
+        if (n_chunks > 1) {
+            BR_CUDA(cudaEventRecord(ctx->pipe_ev[8 + c], s_k));
+            BR_CUDA(cudaStreamWaitEvent(s_out, ctx->pipe_ev[8 + c], 0));
+        }
+        for (Blk &b : blks) {
+            if (!b.bytes || !b.out) continue;
+            const size_t row = b.bytes / N;
+            BR_CUDA(cudaMemcpyAsync((char *)b.host + i0 * row, (const char *)*b.dev + i0 * row, (i1 - i0) * row,
+                                    cudaMemcpyDeviceToHost, s_out));
+        }
+    }
+    if (n_chunks > 1) {
+        BR_CUDA(cudaEventRecord(ctx->pipe_ev[17], s_out));
+        BR_CUDA(cudaStreamWaitEvent(st, ctx->pipe_ev[17], 0));
     }
     BR_CUDA(cudaStreamSynchronize(st));
     if (h2d_bytes) *h2d_bytes = up;
@@ -567,6 +613,10 @@ int br_destroy(br_ctx *ctx)
     if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
     if (ctx->graph) cudaGraphDestroy(ctx->graph);
     if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->pipe_ready) {
+        for (int i = 0; i < 3; ++i) cudaStreamDestroy(ctx->pipe[i]);
+        for (int i = 0; i < 2 * 8 + 2; ++i) cudaEventDestroy(ctx->pipe_ev[i]);
+    }
     delete ctx;
     return BR_OK;
 }

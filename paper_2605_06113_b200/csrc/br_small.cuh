@@ -87,7 +87,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
 
 #pragma unroll 1
     for (int it = 0; it < a.n_steps; ++it, ++k) {
-        const size_t orow = (size_t)it * a.N + row;
+        const size_t orow = (size_t)it * a.N + inst;          // outputs use the rows of the state (first_instance = 0 when n_steps > 1)
         int32_t *assign = a.assign_out + orow * W;
 #pragma unroll
         for (int t = 0; t < NT4; ++t) {

@@ -135,3 +135,67 @@ def test_brh_flat_slope_takes_the_full_scan():
     run_parity(wlm.get_config("c2", H=1, alpha=1.0, beta=1.0, gamma=1.0, gate=0.0, delta_T=1), 2, 150,
                check_every=25)
     run_parity(wlm.get_config("c4", H=2, alpha=1.0, beta=1.0, gamma=1.0), 1, 60, check_every=20)
+
+
+@pytest.mark.parametrize("name,n_inst", [("c3", 600), ("c3", 2100), ("c2", 520)])
+def test_host_buffer_step_in_chunks_matches_device_step(name, n_inst):
+    """br_step_host on batches large enough to go through in chunks of instances (uploads, kernels
+    and downloads of different chunks overlap on three streams): state and outputs must equal those
+    of br_step on device buffers, for three steps in a row."""
+    import torch
+    from paper_2605_06113_b200.binding import Router, state_to_numpy
+    cfg = wlm.get_config(name)
+    wl = wlm.make_workload(cfg, n_instances=n_inst)
+    r = Router(wl, device="cuda:0")
+    st_h = {k: np.ascontiguousarray(v).copy() for k, v in wl.state.items()}
+    out_h = {k: v.numpy() for k, v in r.outputs(n_inst, device="cpu").items()}
+    st_d = r.device_state()
+    out_d = r.outputs(n_inst)
+    for k in range(3):
+        probs = np.ascontiguousarray(wlm.term_probs_np(wl, k)) if cfg.H > 0 else None
+        r.step_host(st_h, out_h, probs)
+        r.step(st_d, out_d, None if probs is None else torch.from_numpy(probs).cuda())
+        torch.cuda.synchronize()
+        for key in out_h:
+            assert np.array_equal(out_h[key], out_d[key].cpu().numpy()), (name, k, key)
+        ref = state_to_numpy(st_d)
+        for key in st_h:
+            assert np.array_equal(st_h[key], ref[key]), (name, k, key)
+    r.close()
+
+
+@pytest.mark.parametrize("name", ["c3", "c2"])
+def test_row_offset_batches(name):
+    """first_instance selects a range of rows of every array, state and outputs alike: stepping
+    rows [5, 12) of a 16-row allocation must leave the other rows untouched and give what a
+    7-instance batch of the same seeds gives."""
+    import torch
+    from paper_2605_06113_b200.binding import Router, state_to_numpy
+    cfg = wlm.get_config(name)
+    wl = wlm.make_workload(cfg, n_instances=16)
+    r = Router(wl, device="cuda:0", threads=32 if name == "c3" else 0)
+    st = r.device_state(); out = r.outputs(16)
+    for v in out.values():
+        v.fill_(-9)
+    wl7 = wlm.make_workload(cfg, n_instances=7, first_instance=5)
+    r7 = Router(wl7, device="cuda:0", threads=32 if name == "c3" else 0)
+    st7 = r7.device_state(); out7 = r7.outputs(7)
+    before = state_to_numpy({k: v.clone() for k, v in st.items()})
+    for k in range(3):
+        probs16 = probs7 = None
+        if cfg.H > 0:
+            probs16 = torch.from_numpy(wlm.term_probs_np(wl, k)).cuda()
+            probs7 = torch.from_numpy(wlm.term_probs_np(wl7, k)).cuda()
+        r.step(st, out, probs16, N=7, first=5)
+        r7.step(st7, out7, probs7)
+        torch.cuda.synchronize()
+        for key in out7:
+            assert torch.equal(out[key][0, 5:12], out7[key][0]), (name, k, key)
+            assert bool((out[key][0, :5] == -9).all()) and bool((out[key][0, 12:] == -9).all()), (name, k, key)
+    after = state_to_numpy(st); ref = state_to_numpy(st7)
+    for key in after:
+        if key == "seed":
+            continue
+        assert np.array_equal(after[key][5:12], ref[key]), key
+        assert np.array_equal(after[key][:5], before[key][:5]) and np.array_equal(after[key][12:], before[key][12:]), key
+    r.close(); r7.close()
