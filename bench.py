@@ -457,9 +457,9 @@ def run_ours(args):
         except Exception as ex:  # keep the headline line even if an extra fails
             line["extra"] = {"error": repr(ex)}
         # ---------------- CPU baseline: the checker on host cores ----------------
-        rate, done, dt = oracle_rate("c3", 12.0, 512, 500)
+        rate, done, dt = oracle_rate("c3", 20.0, 1024, 500)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{done} instance-steps of c3 (first 512 instances, steps 0..{done // 512 - 1}), "
+                                "sample": f"{done} instance-steps of c3 (first 1024 instances, steps 0..{done // 1024 - 1}), "
                                           f"{dt:.1f} s, single thread"}
     elif rank == 0:
         line["e2e"] = None
