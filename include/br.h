@@ -239,6 +239,21 @@ int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int
 int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *win, int32_t R,
                    const int64_t *margins, const int32_t *lim, uint32_t *best_mask, double *best_F);
 
+/*
+ * Pool-bypass dispatch for BR-0 (Appendix "Pool-bypass deployment path for BR-0"; ctx must have
+ * H = 0, else BR_EINVAL).  For each instance the n_requests prompt lengths s [N][n_requests] are
+ * routed one at a time in arrival order: request i goes to argmax_g F_g(s_i) (Eq. 1 with the
+ * context's coefficients, lowest g on ties) over the workers with inflight[g] < inflight_cap[g],
+ * where the margins m_g = M - L_g come from the virtual loads virtual_load [N][G] (running plus
+ * dispatched-but-not-yet-running requests).  The chosen worker's virtual load grows by s_i and its
+ * inflight count by one before the next request is scored.  worker_out [N][n_requests] receives
+ * the worker, -1 when every worker is at its cap; virtual_load and inflight are updated in place.
+ * Device pointers, asynchronous on batch.stream.
+ */
+int br_bypass_dispatch(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int32_t n_requests,
+                       int64_t *virtual_load, int32_t *inflight, const int32_t *inflight_cap,
+                       int32_t *worker_out);
+
 /* Frees the context, its staging buffers and graph.  NULL is accepted. */
 int br_destroy(br_ctx *ctx);
 

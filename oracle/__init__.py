@@ -78,6 +78,8 @@ def lib():
         L.orc_best_subset.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
                                       C.c_double, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_void_p]
+        L.orc_bypass.argtypes = [C.c_int32, C.c_int32, C.c_double, C.c_double, C.c_void_p, C.c_int32,
+                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -143,6 +145,18 @@ def best_subset(score_mode, G, H, alpha, beta, gamma, m, win, lim):
     mask = lib().orc_best_subset(score_mode, G, H, alpha, beta, gamma, _p(mm), _p(ww), len(ww),
                                  lim, C.addressof(f))
     return int(mask), float(f.value)
+
+
+def bypass(G, s, vload, inflight, cap, score_mode=0, alpha=1.0, beta=None):
+    """Pool-bypass dispatch of the requests s in order; returns (workers, virtual loads, inflight)."""
+    ss = np.ascontiguousarray(s, dtype=np.int32)
+    L = np.ascontiguousarray(vload, dtype=np.int64).copy()
+    n = np.ascontiguousarray(inflight, dtype=np.int32).copy()
+    c = np.ascontiguousarray(cap, dtype=np.int32)
+    out = np.zeros(len(ss), dtype=np.int32)
+    lib().orc_bypass(G, score_mode, alpha, float(G) if beta is None else beta, _p(ss), len(ss), _p(L), _p(n),
+                     _p(c), _p(out))
+    return out, L, n
 
 
 # ---- one routing instance --------------------------------------------------

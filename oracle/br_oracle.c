@@ -662,3 +662,30 @@ void orc_projection(orc_inst *s, int64_t *Lh, int64_t *Mh, int64_t *m)
 
 /* PREDICT alone (for the refresh-rule tests) */
 void orc_predict_only(orc_inst *s, const float *probs) { predict(s, probs); }
+
+/*
+ * Pool-bypass dispatch for BR-0 (Appendix "Pool-bypass deployment path for BR-0"): requests go
+ * one at a time, in arrival order, to argmax_g F_g(s) = alpha s - beta (s - m_g)_+ over the
+ * workers below their inflight cap, with m_g = M - L_g from the virtual loads; the chosen
+ * worker's virtual load and inflight count grow before the next request is scored.
+ * READING: lowest g on ties.  score_mode 0: Eq. 1 with (1, G) in integers; 1: fp64 with (alpha, beta).
+ */
+void orc_bypass(int32_t G, int32_t score_mode, double alpha, double beta, const int32_t *s,
+                int32_t n_req, int64_t *vload, int32_t *inflight, const int32_t *cap, int32_t *g_out)
+{
+    for (int i = 0; i < n_req; ++i) {
+        int64_t M = vload[0];
+        for (int g = 1; g < G; ++g) if (vload[g] > M) M = vload[g];
+        int best = -1; double fb = 0.0;
+        for (int g = 0; g < G; ++g) {
+            if (inflight[g] >= cap[g]) continue;
+            int64_t m = M - vload[g];
+            double d1 = 1.0;
+            double f = score_mode == 0 ? (double)orc_f_br0(G, s[i], m)
+                                       : orc_f_brh(0, alpha, beta, &d1, 1.0, s[i], &m);
+            if (best < 0 || f > fb) { best = g; fb = f; }
+        }
+        g_out[i] = best;
+        if (best >= 0) { vload[best] += s[i]; inflight[best] += 1; }
+    }
+}

@@ -55,7 +55,7 @@ class BrLoadOut(C.Structure):
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
            "br_step_host_static",
-           "br_fscore", "br_best_subset", "br_destroy", "br_strerror", "br_version"]
+           "br_fscore", "br_best_subset", "br_bypass_dispatch", "br_destroy", "br_strerror", "br_version"]
 
 _lib = None
 
@@ -87,6 +87,8 @@ def lib():
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_best_subset.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.br_bypass_dispatch.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_destroy.argtypes = [C.c_void_p]
         L.br_strerror.restype = C.c_char_p
         L.br_strerror.argtypes = [C.c_int]
@@ -267,6 +269,14 @@ class Router:
         if rc != BR_OK:
             raise BrError(rc, "br_fscore")
 
+
+    def bypass_dispatch(self, s, virtual_load, inflight, inflight_cap, worker_out, N=None, first=0, stream=None):
+        N = s.shape[0] - first if N is None else N
+        b = BrInstanceBatch(n_instances=N, first_instance=first, n_steps=1, stream=self._stream(stream))
+        rc = lib().br_bypass_dispatch(self._h, C.byref(b), _ptr(s), int(s.shape[1]), _ptr(virtual_load),
+                                      _ptr(inflight), _ptr(inflight_cap), _ptr(worker_out))
+        if rc != BR_OK:
+            raise BrError(rc, "br_bypass_dispatch")
 
     def best_subset(self, win, margins, lim, best_mask, best_F=None, N=None, first=0, stream=None):
         N = win.shape[0] - first if N is None else N

@@ -11,6 +11,7 @@
 #include "br_small.cuh"
 #include "br_fscore.cuh"
 #include "br_subset.cuh"
+#include "br_bypass.cuh"
 
 using br::StepArgs;
 
@@ -604,6 +605,30 @@ int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *w
     br::br_subset_kernel<<<batch->n_instances, 256, 0, (cudaStream_t)batch->stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_best_subset launch");
+    return BR_OK;
+}
+
+int br_bypass_dispatch(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int32_t n_requests,
+                       int64_t *virtual_load, int32_t *inflight, const int32_t *inflight_cap, int32_t *worker_out)
+{
+    if (!ctx || !batch || !s || !virtual_load || !inflight || !inflight_cap || !worker_out) return BR_EINVAL;
+    if (ctx->H != 0) return BR_EINVAL;                       // the pool-bypass path exists for BR-0 only
+    if (batch->n_instances < 0 || batch->first_instance < 0 || n_requests < 0) return BR_EINVAL;
+    if (misaligned(s, 4) || misaligned(virtual_load, 8) || misaligned(inflight, 4) ||
+        misaligned(inflight_cap, 4) || misaligned(worker_out, 4))
+        return BR_EINVAL;
+    if (batch->n_instances == 0 || n_requests == 0) return BR_OK;
+    br::BypassArgs a;
+    memset(&a, 0, sizeof(a));
+    a.f.G = ctx->G; a.f.H = 0; a.f.fp = ctx->p.score_mode == 1;
+    a.f.aD = ctx->base.aD; a.f.beta = ctx->base.beta;
+    for (int h = 0; h <= BR_MAX_H; ++h) a.f.d[h] = ctx->base.d[h];
+    a.n_req = n_requests; a.first_instance = batch->first_instance;
+    a.s = s; a.vload = virtual_load; a.inflight = inflight; a.cap = inflight_cap; a.g_out = worker_out;
+    const int blocks = (batch->n_instances + 3) / 4;
+    br::br_bypass_kernel<<<blocks, 128, 0, (cudaStream_t)batch->stream>>>(a, batch->n_instances);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "br_bypass_dispatch launch");
     return BR_OK;
 }
 

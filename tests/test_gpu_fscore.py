@@ -46,3 +46,34 @@ def test_fscore_matrix_and_best_worker(name, H):
             want = -1 if len(ok) == 0 else int(ok[np.argmax(ref[ok])])
             assert bh[n, i] == want
     r.close()
+
+
+@pytest.mark.parametrize("G,score_mode", [(32, 0), (64, 0), (5, 0), (16, 1)])
+def test_pool_bypass_dispatch(G, score_mode):
+    """br_bypass_dispatch against the checker: workers, virtual loads and inflight counts."""
+    kw = dict(G=G, init_active=8, init_queue=0)
+    if score_mode == 1:
+        kw.update(score_mode=1, alpha=1.0, beta=7.5, gamma=1.0)
+    cfg = wlm.get_config("c3", **kw)
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device="cuda:0")
+    rng = np.random.default_rng(71 + G)
+    N, n_req = 9, 150
+    s = rng.integers(1, 40000, (N, n_req)).astype(np.int32)
+    s[0] = 1000                                            # equal lengths: ties between workers
+    L = rng.integers(0, 300000, (N, G)).astype(np.int64)
+    L[1] = 5000                                            # equal loads
+    infl = rng.integers(0, 10, (N, G)).astype(np.int32)
+    cap = rng.integers(8, 14, (N, G)).astype(np.int32)     # tight caps: some instances fill up
+    cap[2] = 0
+    st, Lt, it, ct = (torch.from_numpy(x.copy()).cuda() for x in (s, L, infl, cap))
+    out = torch.full((N, n_req), -7, dtype=torch.int32, device="cuda")
+    r.bypass_dispatch(st, Lt, it, ct, out)
+    torch.cuda.synchronize()
+    for n in range(N):
+        want, Lw, nw = oracle.bypass(G, s[n], L[n], infl[n], cap[n], score_mode=score_mode, alpha=cfg.alpha,
+                                     beta=float(G) if score_mode == 0 else cfg.beta)
+        assert np.array_equal(out[n].cpu().numpy(), want), n
+        assert np.array_equal(Lt[n].cpu().numpy(), Lw) and np.array_equal(it[n].cpu().numpy(), nw), n
+    assert (out[2] == -1).all()
+    r.close()

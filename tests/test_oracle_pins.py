@@ -681,3 +681,34 @@ def test_eq2_single_request_argmax_sits_next_to_the_peak():
                     assert fb > fa
                 elif a_ >= sstar:
                     assert fb < fa
+
+
+def test_pool_bypass_sends_each_request_where_imbalance_grows_least():
+    """Pool-bypass BR-0 (Appendix "Pool-bypass deployment path for BR-0"): each request goes to
+    argmax_g F_g(s) on the virtual loads, and F = -Delta I (Section 3.1), so the chosen worker is
+    the one whose admission raises I = G max L - sum L the least among the workers below their
+    inflight cap (lowest g on ties); loads and inflight counts move before the next request."""
+    rng = np.random.default_rng(59)
+    for _ in range(40):
+        G = int(rng.integers(1, 12)); n = int(rng.integers(1, 30))
+        L = rng.integers(0, 3000, G).astype(np.int64)
+        infl = rng.integers(0, 4, G).astype(np.int32)
+        cap = rng.integers(1, 7, G).astype(np.int32)
+        s = rng.integers(1, 1500, n).astype(np.int32)
+        got, L_out, n_out = oracle.bypass(G, s, L, infl, cap)
+        Lr, nr = L.copy(), infl.copy()
+        for i in range(n):
+            ok = [g for g in range(G) if nr[g] < cap[g]]
+            if not ok:
+                assert got[i] == -1
+                continue
+            def grow(g):
+                after = Lr.copy(); after[g] += s[i]
+                return oracle.imbalance(after) - oracle.imbalance(Lr)
+            want = min(ok, key=lambda g: (grow(g), g))
+            assert got[i] == want
+            Lr[want] += s[i]; nr[want] += 1
+        assert np.array_equal(L_out, Lr) and np.array_equal(n_out, nr)
+    # one worker, or everything at its cap
+    got, _, _ = oracle.bypass(1, [5, 6], [10], [0], [1])
+    assert list(got) == [0, -1]
