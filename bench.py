@@ -505,10 +505,86 @@ def extras(torch, device, args, peak):
                          "frac": m["achieved"] / peak, "traffic": recorded_traffic("c4", spl),
                          "algorithmic_bytes_per_launch": m["abytes_per_launch"],
                          "kernel": kernel_name("c4")}}
+    # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
+    try:
+        ex["entry_points"] = entry_points(torch, device, peak)
+    except Exception as e:
+        ex["entry_points"] = {"error": repr(e)}
     # latency path: one instance, one graph-replayed step per decode step
     ex["latency"] = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
                      latency_path(torch, "c4", device, 1000)]
     return ex
+
+
+def _time_call(torch, fn, reps=20, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def entry_points(torch, device, peak):
+    """Timings of br_fscore (HBM-bound: the matrix is written once), br_bypass_dispatch and
+    br_best_subset on synthetic inputs of the c3 / c4 shapes."""
+    from paper_2605_06113_b200.binding import Router
+    res = {}
+    gen = torch.Generator(device=device); gen.manual_seed(7)
+    # F-score matrix: c4 shape, 1024 instances x 1024 requests x 64 workers in fp64 (512 MB out)
+    cfg = wlm.get_config("c4")
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device=device)
+    N, n_req, G, H = 1024, 1024, cfg.G, cfg.H
+    s = torch.randint(1, 60000, (N, n_req), dtype=torch.int32, device=device, generator=gen)
+    Lh = torch.randint(100000, 400000, (N, G, H + 1), dtype=torch.int64, device=device, generator=gen)
+    F = torch.empty((N, n_req, G), dtype=torch.float64, device=device)
+    ms = _time_call(torch, lambda: r.fscore(s, Lh, F))
+    byt = F.numel() * 8 + s.numel() * 4 + Lh.numel() * 8
+    res["br_fscore"] = {"workload": "c4 shape (Eq. 2, H=8): 1024 instances x 1024 requests x 64 workers, fp64 matrix",
+                        "ms": ms, "scores_per_s": F.numel() / (ms * 1e-3),
+                        "roofline": {"bound": "hbm", "achieved": byt / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                     "frac": byt / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                                     "algorithmic_bytes_per_launch": byt, "kernel": "br_fscore_kernel"}}
+    del F
+    r.close()
+    # pool-bypass dispatch and subset solver: c3 shape (Eq. 1)
+    cfg = wlm.get_config("c3")
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device=device)
+    N, n_req, G = 4096, 256, cfg.G
+    s = torch.randint(1, 40000, (N, n_req), dtype=torch.int32, device=device, generator=gen)
+    L0 = torch.randint(0, 300000, (N, G), dtype=torch.int64, device=device, generator=gen)
+    F = torch.empty((N, 1024, G), dtype=torch.float64, device=device)
+    s4 = torch.randint(1, 40000, (N, 1024), dtype=torch.int32, device=device, generator=gen)
+    ms = _time_call(torch, lambda: r.fscore(s4, L0.view(N, G, 1), F))
+    byt = F.numel() * 8 + s4.numel() * 4 + L0.numel() * 8
+    res["br_fscore_eq1"] = {"workload": "c3 shape (Eq. 1): 4096 instances x 1024 requests x 32 workers, fp64 matrix",
+                            "ms": ms, "scores_per_s": F.numel() / (ms * 1e-3),
+                            "roofline": {"bound": "hbm", "achieved": byt / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                         "frac": byt / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                                         "algorithmic_bytes_per_launch": byt, "kernel": "br_fscore_kernel<0>"}}
+    del F, s4
+    cap = torch.full((N, G), 1 << 30, dtype=torch.int32, device=device)
+    L = L0.clone(); infl = torch.zeros((N, G), dtype=torch.int32, device=device)
+    out = torch.empty((N, n_req), dtype=torch.int32, device=device)
+    ms = _time_call(torch, lambda: r.bypass_dispatch(s, L, infl, cap, out))
+    res["br_bypass_dispatch"] = {"workload": "c3 shape: 4096 instances, 256 requests each dispatched in order over 32 workers",
+                                 "ms": ms, "requests_per_s": N * n_req / (ms * 1e-3)}
+    R, P = 16, 4096
+    win = torch.randint(1, 40000, (P, R), dtype=torch.int32, device=device, generator=gen)
+    m = torch.randint(0, 200000, (P, 1), dtype=torch.int64, device=device, generator=gen)
+    lim = torch.full((P,), R, dtype=torch.int32, device=device)
+    mask = torch.empty((P,), dtype=torch.int32, device=device)
+    ms = _time_call(torch, lambda: r.best_subset(win, m, lim, mask))
+    res["br_best_subset"] = {"workload": "4096 problems, window of 16 requests (65,535 subsets each), Eq. 1",
+                             "ms": ms, "problems_per_s": P / (ms * 1e-3), "subsets_per_s": P * ((1 << R) - 1) / (ms * 1e-3)}
+    r.close()
+    return res
 
 
 def main():

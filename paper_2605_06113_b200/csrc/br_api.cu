@@ -580,7 +580,9 @@ int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int
     a.s = s; a.Lh = Lh; a.cap = cap; a.F = F; a.best_g = best_g;
     const int tiles = (n_requests + br::kFsTile - 1) / br::kFsTile;
     dim3 grid(tiles, batch->n_instances);
-    br::br_fscore_kernel<<<grid, 256, 0, (cudaStream_t)batch->stream>>>(a);
+    void (*kern)(const br::FscoreArgs) = ctx->H == 0 ? br::br_fscore_kernel<0> : ctx->H <= 4 ? br::br_fscore_kernel<4>
+                                       : ctx->H <= 8 ? br::br_fscore_kernel<8> : br::br_fscore_kernel<16>;
+    kern<<<grid, 256, 0, (cudaStream_t)batch->stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_fscore launch");
     return BR_OK;

@@ -39,13 +39,18 @@ __device__ __forceinline__ long long fscore_key(const FscoreArgs &a, int delta, 
     return key_of_double(__dsub_rn(__dmul_rn(a.aD, dl), __dmul_rn(a.beta, pen)));
 }
 
+// Thread t of a block owns worker g = t % G for the whole tile (its margins and discounts stay in
+// registers) and walks the requests slice, slice + n_slices, ...: thread t writes elements
+// t, t + n_slices * G, ... of the tile's [request][worker] rows, so every store instruction of a
+// warp covers consecutive addresses.  HM bounds H at compile time (loops over h unrolled).
+template <int HM>
 __global__ void __launch_bounds__(256) br_fscore_kernel(const FscoreArgs a)
 {
     __shared__ long long m_s[BR_MAX_G * (BR_MAX_H + 1)];
     __shared__ long long Mh[BR_MAX_H + 1];
     __shared__ __align__(16) int s_tile[kFsTile];
     __shared__ int cap_s[BR_MAX_G];
-    const int tid = threadIdx.x, G = a.G, H1 = a.H + 1;
+    const int tid = threadIdx.x, G = a.G, H = a.H, H1 = a.H + 1;
     const size_t inst = (size_t)a.first_instance + blockIdx.y;
     const int tile0 = blockIdx.x * kFsTile;
     const int n = min(kFsTile, a.n_req - tile0);
@@ -66,10 +71,43 @@ __global__ void __launch_bounds__(256) br_fscore_kernel(const FscoreArgs a)
     __syncthreads();
 
     double *F = a.F + (inst * a.n_req + tile0) * G;
-    for (int o = tid; o < n * G; o += blockDim.x) {
-        const int i = o / G, g = o - i * G;
-        const long long key = fscore_key(a, s_tile[i], m_s + g * H1);
-        F[o] = a.fp ? double_of_key(key) : (double)key;
+    const int n_slices = blockDim.x / G;
+    const int slice = tid / G, g = tid - slice * G;
+    if (slice < n_slices) {
+        double md[HM + 1], dd[HM + 1];
+        long long m0 = m_s[g * H1], mmin = m0;
+#pragma unroll
+        for (int h = 0; h <= HM; ++h) {
+            md[h] = h <= H ? (double)m_s[g * H1 + h] : 0.0;
+            dd[h] = h <= H ? a.d[h] : 0.0;
+            if (h <= H) mmin = min(mmin, m_s[g * H1 + h]);
+        }
+        const long long Gl = (long long)G;
+#pragma unroll 4
+        for (int i = slice; i < n; i += n_slices) {
+            const int si = s_tile[i];
+            double f;
+            if (!a.fp) {
+                long long over = (long long)si - m0;
+                over = over > 0 ? over : 0;
+                f = (double)((long long)si - Gl * over);                    // Eq. 1, exact
+            } else {
+                const double dl = (double)si;
+                double pen = 0.0;
+                if ((long long)si > mmin) {                                 // else every (s - m_h)_+ is zero
+#pragma unroll
+                    for (int h = 0; h <= HM; ++h) {
+                        if (h <= H) {
+                            double over = __dsub_rn(dl, md[h]);
+                            over = over > 0.0 ? over : 0.0;
+                            pen = __dadd_rn(pen, __dmul_rn(dd[h], over));
+                        }
+                    }
+                }
+                f = __dsub_rn(__dmul_rn(a.aD, dl), __dmul_rn(a.beta, pen)) + 0.0;   // Eq. 2 (-0.0 -> +0.0)
+            }
+            F[(size_t)i * G + g] = f;
+        }
     }
     if (a.best_g) {
         for (int i = tid; i < n; i += blockDim.x) {
