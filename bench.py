@@ -584,6 +584,18 @@ def entry_points(torch, device, peak):
     res["br_best_subset"] = {"workload": "4096 problems, window of 16 requests (65,535 subsets each), Eq. 1",
                              "ms": ms, "problems_per_s": P / (ms * 1e-3), "subsets_per_s": P * ((1 << R) - 1) / (ms * 1e-3)}
     r.close()
+    # empirical-survival estimator: 4M requests against a history of 1M output lengths (H = 8)
+    cfg = wlm.get_config("c4")
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device=device)
+    hist = torch.sort(torch.randint(1, 4000, (1 << 20,), dtype=torch.int32, device=device, generator=gen)).values
+    prefix = torch.cat([torch.zeros(1, dtype=torch.int64, device=device), torch.cumsum(hist.to(torch.int64), 0)])
+    age = torch.randint(0, 4000, (1 << 22,), dtype=torch.int32, device=device, generator=gen)
+    c = torch.empty(age.numel(), dtype=torch.float32, device=device)
+    ms = _time_call(torch, lambda: r.survival_chat(hist, prefix, age, c))
+    res["br_survival_chat"] = {"workload": "4,194,304 requests, history of 1,048,576 output lengths, H = 8",
+                               "ms": ms, "requests_per_s": age.numel() / (ms * 1e-3)}
+    r.close()
     return res
 
 

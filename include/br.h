@@ -254,6 +254,21 @@ int br_bypass_dispatch(br_ctx *ctx, const br_instance_batch *batch, const int32_
                        int64_t *virtual_load, int32_t *inflight, const int32_t *inflight_cap,
                        int32_t *worker_out);
 
+/*
+ * Empirical-survival estimator of c_hat (Appendix "Estimator realizations", "Empirical-survival";
+ * Eqs. 3-5), for contexts with H >= 1.  hist_sorted [n_hist] holds recorded output lengths in
+ * ascending order, hist_prefix [n_hist + 1] their prefix sums (hist_prefix[j] = sum of the first
+ * j entries).  For each of count requests with age[i] tokens produced so far:
+ *   p_fin = #{age < o <= age + H} / #{o > age},  mu_rem = mean of (o - age) over that window,
+ *   c_hat = (1 - p_fin) H + p_fin mu_rem clipped to [0, H]   (fp64, stored as fp32);
+ * with no recorded output inside the window p_fin = 0, mu_rem = H and c_hat = H.  p_fin and
+ * mu_rem [count] may be NULL.  Device pointers; asynchronous on stream (a cudaStream_t).
+ * BR_EINVAL for null pointers, H = 0, n_hist < 1 or count < 0.
+ */
+int br_survival_chat(br_ctx *ctx, void *stream, const int32_t *hist_sorted, const int64_t *hist_prefix,
+                     int32_t n_hist, const int32_t *age, int64_t count, float *c_hat, double *p_fin,
+                     double *mu_rem);
+
 /* Frees the context, its staging buffers and graph.  NULL is accepted. */
 int br_destroy(br_ctx *ctx);
 

@@ -80,6 +80,8 @@ def lib():
                                       C.c_void_p]
         L.orc_bypass.argtypes = [C.c_int32, C.c_int32, C.c_double, C.c_double, C.c_void_p, C.c_int32,
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.orc_survival.restype = C.c_double
+        L.orc_survival.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -145,6 +147,14 @@ def best_subset(score_mode, G, H, alpha, beta, gamma, m, win, lim):
     mask = lib().orc_best_subset(score_mode, G, H, alpha, beta, gamma, _p(mm), _p(ww), len(ww),
                                  lim, C.addressof(f))
     return int(mask), float(f.value)
+
+
+def survival(hist, H, age):
+    """Empirical-survival (c_hat, p_fin, mu_rem) of a request of the given age."""
+    h = np.ascontiguousarray(hist, dtype=np.int32)
+    p = C.c_double(); mu = C.c_double()
+    c = lib().orc_survival(_p(h), len(h), int(H), int(age), C.addressof(p), C.addressof(mu))
+    return float(c), float(p.value), float(mu.value)
 
 
 def bypass(G, s, vload, inflight, cap, score_mode=0, alpha=1.0, beta=None):

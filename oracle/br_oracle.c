@@ -19,6 +19,8 @@
  *   refresh period, confidence gate, floor ........................ Appendix "Refresh logic"
  *   exhaustive subset enumeration over the R_max window ........... Appendix "Bit-set subset selection"
  *   round-robin and least-loaded comparison routers ............... Section 5.1 "Baselines"
+ *   pool-bypass dispatch of BR-0 .................................. Appendix "Pool-bypass deployment path for BR-0"
+ *   empirical-survival estimator of c_hat ......................... Appendix "Estimator realizations"
  *
  * Readings taken where the paper is silent or ambiguous are marked READING
  * below.  Functions whose tie-break choices have no counterpart in the paper
@@ -688,4 +690,32 @@ void orc_bypass(int32_t G, int32_t score_mode, double alpha, double beta, const 
         g_out[i] = best;
         if (best >= 0) { vload[best] += s[i]; inflight[best] += 1; }
     }
+}
+
+/*
+ * Empirical-survival estimator (Appendix "Estimator realizations", "Empirical-survival"), written
+ * from its definition by counting over the history (any order):
+ *   p_fin = #{a < o_j <= a + H} / #{o_j > a},  mu_rem = mean of (o_j - a) over that window,
+ *   c_hat = (1 - p_fin) H + p_fin mu_rem  (Eq. 5), clipped to [0, H].
+ * READING: with no recorded output inside the window (in particular when the request is older
+ * than every recorded output) p_fin = 0, mu_rem = H, c_hat = H (the conservative anchor).
+ */
+double orc_survival(const int32_t *hist, int32_t n, int32_t H, int32_t age, double *p_fin, double *mu_rem)
+{
+    int64_t c0 = 0, c1 = 0, sum1 = 0;
+    for (int j = 0; j < n; ++j) {
+        if (hist[j] > age) ++c0;
+        if (hist[j] > age && (int64_t)hist[j] <= (int64_t)age + H) { ++c1; sum1 += (int64_t)hist[j] - age; }
+    }
+    double p = 0.0, mu = (double)H, c = (double)H;
+    if (c1 > 0) {
+        p = (double)c1 / (double)c0;
+        mu = (double)sum1 / (double)c1;
+        c = (1.0 - p) * (double)H + p * mu;
+        if (c < 0.0) c = 0.0;
+        if (c > (double)H) c = (double)H;
+    }
+    if (p_fin) *p_fin = p;
+    if (mu_rem) *mu_rem = mu;
+    return c;
 }

@@ -55,7 +55,7 @@ class BrLoadOut(C.Structure):
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
            "br_step_host_static",
-           "br_fscore", "br_best_subset", "br_bypass_dispatch", "br_destroy", "br_strerror", "br_version"]
+           "br_fscore", "br_best_subset", "br_bypass_dispatch", "br_survival_chat", "br_destroy", "br_strerror", "br_version"]
 
 _lib = None
 
@@ -89,6 +89,8 @@ def lib():
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_bypass_dispatch.argtypes = [C.c_void_p, C.POINTER(BrInstanceBatch), C.c_void_p, C.c_int32,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.br_survival_chat.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                       C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_destroy.argtypes = [C.c_void_p]
         L.br_strerror.restype = C.c_char_p
         L.br_strerror.argtypes = [C.c_int]
@@ -277,6 +279,13 @@ class Router:
                                       _ptr(inflight), _ptr(inflight_cap), _ptr(worker_out))
         if rc != BR_OK:
             raise BrError(rc, "br_bypass_dispatch")
+
+    def survival_chat(self, hist_sorted, hist_prefix, age, c_hat, p_fin=None, mu_rem=None, stream=None):
+        rc = lib().br_survival_chat(self._h, self._stream(stream), _ptr(hist_sorted), _ptr(hist_prefix),
+                                    int(hist_sorted.numel()), _ptr(age), int(age.numel()), _ptr(c_hat),
+                                    _ptr(p_fin), _ptr(mu_rem))
+        if rc != BR_OK:
+            raise BrError(rc, "br_survival_chat")
 
     def best_subset(self, win, margins, lim, best_mask, best_F=None, N=None, first=0, stream=None):
         N = win.shape[0] - first if N is None else N

@@ -12,6 +12,7 @@
 #include "br_fscore.cuh"
 #include "br_subset.cuh"
 #include "br_bypass.cuh"
+#include "br_survival.cuh"
 
 using br::StepArgs;
 
@@ -631,6 +632,27 @@ int br_bypass_dispatch(br_ctx *ctx, const br_instance_batch *batch, const int32_
     br::br_bypass_kernel<<<blocks, 128, 0, (cudaStream_t)batch->stream>>>(a, batch->n_instances);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_bypass_dispatch launch");
+    return BR_OK;
+}
+
+int br_survival_chat(br_ctx *ctx, void *stream, const int32_t *hist_sorted, const int64_t *hist_prefix,
+                     int32_t n_hist, const int32_t *age, int64_t count, float *c_hat, double *p_fin,
+                     double *mu_rem)
+{
+    if (!ctx || !hist_sorted || !hist_prefix || !age || !c_hat) return BR_EINVAL;
+    if (ctx->H < 1 || n_hist < 1 || count < 0) return BR_EINVAL;
+    if (misaligned(hist_sorted, 4) || misaligned(hist_prefix, 8) || misaligned(age, 4) || misaligned(c_hat, 4) ||
+        (p_fin && misaligned(p_fin, 8)) || (mu_rem && misaligned(mu_rem, 8)))
+        return BR_EINVAL;
+    if (count == 0) return BR_OK;
+    br::SurvivalArgs a;
+    a.hist = hist_sorted; a.prefix = hist_prefix; a.n_hist = n_hist; a.H = ctx->H;
+    a.age = age; a.count = count; a.c_hat = c_hat; a.p_fin = p_fin; a.mu_rem = mu_rem;
+    const int64_t blocks = (count + 255) / 256;
+    if (blocks > 0x7FFFFFFF) return BR_EINVAL;
+    br::br_survival_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "br_survival_chat launch");
     return BR_OK;
 }
 

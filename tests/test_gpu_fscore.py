@@ -77,3 +77,27 @@ def test_pool_bypass_dispatch(G, score_mode):
         assert np.array_equal(Lt[n].cpu().numpy(), Lw) and np.array_equal(it[n].cpu().numpy(), nw), n
     assert (out[2] == -1).all()
     r.close()
+
+
+def test_empirical_survival_estimator():
+    """br_survival_chat against the checker's counting definition (same fp64 operations: equality)."""
+    cfg = wlm.get_config("c4")                              # H = 8
+    wl = wlm.make_workload(cfg, n_instances=1)
+    r = Router(wl, device="cuda:0")
+    rng = np.random.default_rng(83)
+    hist = np.sort(rng.geometric(1 / 600.0, 5000).astype(np.int32))
+    prefix = np.concatenate([[0], np.cumsum(hist.astype(np.int64))]).astype(np.int64)
+    age = np.concatenate([rng.integers(0, 3000, 3000), [0, int(hist[-1]) - 1, int(hist[-1]), int(hist[-1]) + 9,
+                                                        int(hist[0]) - 1, int(hist[0])]]).astype(np.int32)
+    ht, pt, at = (torch.from_numpy(x).cuda() for x in (hist, prefix, age))
+    c = torch.empty(len(age), dtype=torch.float32, device="cuda")
+    p = torch.empty(len(age), dtype=torch.float64, device="cuda")
+    mu = torch.empty(len(age), dtype=torch.float64, device="cuda")
+    r.survival_chat(ht, pt, at, c, p, mu)
+    torch.cuda.synchronize()
+    ch, ph, mh = c.cpu().numpy(), p.cpu().numpy(), mu.cpu().numpy()
+    shuffled = rng.permutation(hist)                        # the definition does not need the order
+    for i in list(range(400)) + list(range(len(age) - 6, len(age))):
+        wc, wp, wm = oracle.survival(shuffled, cfg.H, int(age[i]))
+        assert ch[i] == np.float32(wc) and ph[i] == wp and mh[i] == wm, i
+    r.close()

@@ -712,3 +712,30 @@ def test_pool_bypass_sends_each_request_where_imbalance_grows_least():
     # one worker, or everything at its cap
     got, _, _ = oracle.bypass(1, [5, 6], [10], [0], [1])
     assert list(got) == [0, -1]
+
+
+def test_empirical_survival_estimator_is_the_truncated_expectation():
+    """The empirical-survival c_hat is Eq. 3 on the empirical distribution: the two-stage form
+    (1 - p_fin) H + p_fin mu_rem (Eqs. 4-5) must equal E[min(o - a, H) | o > a] taken directly over
+    the history, in exact rationals; plus the closed forms of a one-point history."""
+    from fractions import Fraction
+    rng = np.random.default_rng(61)
+    for _ in range(60):
+        n = int(rng.integers(1, 200)); H = int(rng.integers(1, 17))
+        hist = rng.integers(1, 120, n)
+        for age in [0, 1, int(rng.integers(0, 130)), int(hist.max()) - 1, int(hist.max()), int(hist.max()) + 5]:
+            c, p, mu = oracle.survival(hist, H, age)
+            alive = [int(o) for o in hist if o > age]
+            inside = [o for o in alive if o <= age + H]
+            if not inside:
+                assert (c, p, mu) == (float(H), 0.0, float(H))
+                # nothing recorded ends inside the window: every survivor contributes the full H
+                continue
+            want = Fraction(sum(min(o - age, H) for o in alive), len(alive))
+            assert abs(Fraction(c) - want) < Fraction(1, 10 ** 12)
+            assert abs(Fraction(p) - Fraction(len(inside), len(alive))) < Fraction(1, 10 ** 14)
+            assert abs(Fraction(mu) - Fraction(sum(o - age for o in inside), len(inside))) < Fraction(1, 10 ** 12)
+            assert 0.0 <= c <= H
+    # one recorded length v: inside the window the request surely ends after v - a more steps
+    assert oracle.survival([50] * 7, 8, 45) == (5.0, 1.0, 5.0)
+    assert oracle.survival([50] * 7, 8, 41)[0] == 8.0 and oracle.survival([50] * 7, 8, 50)[0] == 8.0
