@@ -604,7 +604,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3840)
     ap.add_argument("--warmup", type=int, default=160)
-    ap.add_argument("--steps-per-launch", type=int, default=8,
+    ap.add_argument("--steps-per-launch", type=int, default=16,
                     help="decode steps advanced by one launch (one br_step call with n_steps); used when it divides --steps")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
