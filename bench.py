@@ -428,7 +428,10 @@ def run_ours(args):
         "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
         "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None,
+        # arithmetic of the path: Eq. 1 scores, loads and keys in 32-bit integers (ranges proven at
+        # br_create), 64-bit outputs; the BR-H workload scores Eq. 2 in fp64
+        "dtype": "int32" if wname == "c3" else "f64", "data": "synthetic",
         "config": {"workload": ("c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.." if wname == "c3"
                                 else "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000.."),
                    "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
