@@ -28,6 +28,7 @@ from paper_2605_06113_b200 import workload as wlm  # noqa: E402
 
 METRIC = "routing instance-steps/sec (batched BR-0, 4096 instances, G=32, W=256)"
 UNIT = "instance-steps/s"
+C3_WORKLOAD = "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.."
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -221,7 +222,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
-        "config": {"workload": "c3 (BR-0 batched, G=32, B=64, W=256), 32-instance sample per step"},
+        "config": {"workload": C3_WORKLOAD, "sample": "the first 32 instances, one decode step of each per step"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{n_inst} instances x {args.steps} steps of c3, single thread"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -432,7 +433,7 @@ def run_ours(args):
         # arithmetic of the path: Eq. 1 scores, loads and keys in 32-bit integers (ranges proven at
         # br_create), 64-bit outputs; the BR-H workload scores Eq. 2 in fp64
         "dtype": "int32" if wname == "c3" else "f64", "data": "synthetic",
-        "config": {"workload": ("c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.." if wname == "c3"
+        "config": {"workload": (C3_WORKLOAD if wname == "c3"
                                 else "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000.."),
                    "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
                    "l2": f"{m['n_sets']} instance sets stepped in rotation ({spl} decode steps per launch and "
