@@ -199,3 +199,37 @@ def test_row_offset_batches(name):
         assert np.array_equal(after[key][5:12], ref[key]), key
         assert np.array_equal(after[key][:5], before[key][:5]) and np.array_equal(after[key][12:], before[key][12:]), key
     r.close(); r7.close()
+
+
+def test_small_fleet_random_shapes():
+    """Thirty seeded random fleet shapes inside the small-fleet kernel's range (G <= 32, B <= 64,
+    W <= 512) with random window sizes, stage splits, hazards and arrival rates."""
+    rng = np.random.default_rng(2024)
+    for case in range(30):
+        G = int(rng.integers(1, 33)); B = 8 * int(rng.integers(1, 9)); W = 4 * int(rng.integers(1, 129))
+        cfg = wlm.get_config("c3", G=G, B=B, W=W, R_max=int(rng.integers(1, 6)),
+                             S_greedy=int(rng.choice([-1, 0, 3, G, 4 * G, 1 << 20])),
+                             init_active=int(rng.integers(0, B + 1)), init_queue=int(rng.integers(0, W + 1)),
+                             hazard=float(rng.choice([0.0, 0.002, 0.05, 0.3, 1.0])),
+                             arrival=("const", float(rng.choice([0.01, 1.0, 5.0, 20.0, 45.0]))),
+                             first_seed=1000 * case)
+        run_parity(cfg, 2, 50, threads=32, check_every=10, launch_steps=int(rng.choice([1, 1, 5])))
+
+
+def test_brh_random_shapes():
+    """Seeded random BR-H shapes (H up to 16, G up to 64, ragged B and W), open and closed gates,
+    both termination modes."""
+    rng = np.random.default_rng(4048)
+    for case in range(14):
+        G = int(rng.integers(1, 65)); B = 8 * int(rng.integers(1, 13)); W = 4 * int(rng.integers(1, 151))
+        H = int(rng.integers(1, 17))
+        cfg = wlm.get_config("c2", G=G, B=B, W=W, H=H, R_max=int(rng.integers(1, 6)),
+                             S_greedy=int(rng.choice([-1, 0, G, 1 << 20])), delta_T=int(rng.choice([-1, 1, 2, 5])),
+                             gate=float(rng.choice([0.0, 0.1, 0.5])), beta=float(rng.choice([3.0, 14.67, 43.0])),
+                             gamma=float(rng.choice([0.5, 0.64, 0.9, 1.0])),
+                             init_active=int(rng.integers(0, B + 1)), init_queue=int(rng.integers(0, W + 1)),
+                             term_mode=int(rng.choice([1, 2])), hazard=float(rng.choice([0.002, 0.05, 0.3])),
+                             beta_ab=(2.0, float(rng.choice([4.0, 20.0, 50.0]))),
+                             arrival=("const", float(rng.choice([1.0, 8.0, 30.0]))), first_seed=5000 * case)
+        run_parity(cfg, 2, 40, threads=int(rng.choice([0, 32, 64, 128])), check_every=10,
+                   launch_steps=int(rng.choice([1, 1, 4])))
