@@ -1,4 +1,5 @@
-// The routing-step kernel: one thread block per routing instance.
+// The general routing-step kernel: an instance is served by 32 to 256 threads (BR-H, large fleets,
+// optional outputs; BR-0 on small fleets runs on br_small_kernel).
 //
 // Phases per decode step k (Section 2.2 model; Algorithms 1 and 2):
 //   ARRIVE -> PREDICT (H > 0) -> ROUTE (Stage 1, Stage 2) -> RECORD -> ADVANCE.
@@ -12,7 +13,8 @@
 //
 // Loads are advanced incrementally: L_g(k+1) = L_g(k) - sum of the loads of the requests
 // that end at k + number of survivors, so ADVANCE touches only the occupancy bit masks,
-// one Philox block per 8 slots, and the few slots whose request ends.  Only the horizon
+// one Philox block per worker (the ending slots are walked by geometric gaps), and the few
+// slots whose request ends.  Only the horizon
 // projection of BR-H streams the per-request state.
 #pragma once
 #include "br_device.cuh"
