@@ -57,6 +57,7 @@ def lib():
         L.orc_step.argtypes = [C.c_void_p] + [C.c_void_p] * 5
         L.orc_route_only.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_projection.argtypes = [C.c_void_p] + [C.c_void_p] * 3
+        L.orc_round_projection.argtypes = [C.c_void_p] + [C.c_void_p] * 3
         L.orc_predict_only.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_philox4x32_10.argtypes = [C.c_void_p] * 3
         L.orc_term_gap.restype = C.c_int
@@ -252,6 +253,14 @@ class Instance:
         Lh = np.zeros((self.G, H1), dtype=np.int64); Mh = np.zeros(H1, dtype=np.int64)
         m = np.zeros((self.G, H1), dtype=np.int64)
         lib().orc_projection(self._h, _p(Lh), _p(Mh), _p(m))
+        return Lh, Mh, m
+
+    def round_projection(self):
+        """Projected loads, envelope and margins as the last routing round left them."""
+        H1 = self.H + 1
+        Lh = np.zeros((self.G, H1), dtype=np.int64); Mh = np.zeros(H1, dtype=np.int64)
+        m = np.zeros((self.G, H1), dtype=np.int64)
+        lib().orc_round_projection(self._h, _p(Lh), _p(Mh), _p(m))
         return Lh, Mh, m
 
     def predict_only(self, probs):

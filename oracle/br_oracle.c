@@ -23,11 +23,18 @@
  *   empirical-survival estimator of c_hat ......................... Appendix "Estimator realizations"
  *
  * Readings taken where the paper is silent or ambiguous are marked READING
- * below.  Functions whose tie-break choices have no counterpart in the paper
- * are "parity unpinned" against the paper in that respect only: orc_step's
- * tie-breaks (worker ties, request ties, subset ties) and slot placement.
- * Everything else is pinned by the tests under tests/ (closed forms of Eq. 1,
- * the identity F = -Delta I, the H = 0 reduction, Eq. 4, brute force).
+ * below.  What the paper states is pinned by tests that do not go through this
+ * file's own output: closed forms of Eq. 1, the identity F = -Delta I, the H = 0
+ * reduction, Eq. 4, brute force, and hand-built snapshots for the rules inside
+ * the routing round (worker order of Stage 1 and of the Stage-2 queue, the
+ * horizon-min key, the guard's boundary F <= 0, the constant-s_i update of an
+ * admission over all offsets, the subset choice as the round makes it).
+ * "Parity unpinned" against the paper, because the paper does not state them:
+ * the READINGs themselves -- direction of "sorted by s_i", lowest-index ties
+ * (worker, request, subset mask), the guard's arg-max ranging over all of
+ * R_wait, slot placement, the prediction state given to a new admission.  The
+ * tests fix these readings by hand-built cases too, so a change of one is
+ * noticed, but the paper cannot confirm them.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -657,6 +664,16 @@ void orc_projection(orc_inst *s, int64_t *Lh, int64_t *Mh, int64_t *m)
 {
     int n = s->p.G * (s->p.H + 1);
     project(s);
+    memcpy(Lh, s->Lh, n * sizeof(int64_t));
+    memcpy(Mh, s->Mh, (s->p.H + 1) * sizeof(int64_t));
+    memcpy(m, s->m, n * sizeof(int64_t));
+}
+
+/* The routing round's own projection as it stands (after orc_route_only: the loads, envelope and
+ * margins that the admissions of the round have updated), copied without recomputing anything. */
+void orc_round_projection(const orc_inst *s, int64_t *Lh, int64_t *Mh, int64_t *m)
+{
+    int n = s->p.G * (s->p.H + 1);
     memcpy(Lh, s->Lh, n * sizeof(int64_t));
     memcpy(Mh, s->Mh, (s->p.H + 1) * sizeof(int64_t));
     memcpy(m, s->m, n * sizeof(int64_t));

@@ -1,6 +1,7 @@
 """Builds libbr.so (the C-ABI routing library) in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
+import glob
 import os
 import subprocess
 import sys
@@ -9,7 +10,6 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbr.so")
 SOURCES = ["br_api.cu"]
-HEADERS = ["br_step.cuh", "br_fscore.cuh", "br_device.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -22,8 +22,10 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
+    # every file of csrc/ is a dependency: the kernels live in headers included by br_api.cu
+    deps = glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cuh"))
     deps.append(os.path.join(os.path.dirname(HERE), "include", "br.h"))
+    deps.append(os.path.abspath(__file__))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
