@@ -3,10 +3,16 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-A "step" is one launch of the whole routing path (ARRIVE, PREDICT, ROUTE, RECORD, ADVANCE)
-over one batch of 4,096 independent BR-0 instances (G = 32, 256 waiting each: the batched
-HBM-throughput configuration).  Several instance sets are stepped in rotation so that the
-data touched between two visits of the same set exceeds the L2 cache.  Prints one JSON line.
+A "step" is one call of br_step: one launch of the whole routing path (ARRIVE, PREDICT, ROUTE,
+RECORD, ADVANCE) over one batch of 4,096 independent BR-0 instances (G = 32, 256 waiting each:
+the batched HBM-throughput configuration), advancing every instance by --steps-per-launch
+decode steps (16 unless asked otherwise; `config.steps_per_launch` says which).  The timed
+region of --steps calls is repeated --repeats times, each repeat on instance sets put back to
+their starting snapshots and primed by untimed calls; the median repeat is reported, minimum and
+maximum beside it.  Several instance sets are stepped in rotation so that the data touched
+between two visits of the same set exceeds the L2 cache; they start at evenly spaced points of
+the configuration's trajectory, so that a short timed region still samples all of it.  Prints one JSON line whose last key,
+`summary`, repeats every headline figure in compact form.
 """
 from __future__ import annotations
 
@@ -16,7 +22,6 @@ import os
 import subprocess
 import sys
 import tempfile
-import threading
 import time
 
 import numpy as np
@@ -26,9 +31,15 @@ sys.path.insert(0, ROOT)
 
 from paper_2605_06113_b200 import workload as wlm  # noqa: E402
 
-METRIC = "routing instance-steps/sec (batched BR-0, 4096 instances, G=32, W=256)"
 UNIT = "instance-steps/s"
-C3_WORKLOAD = "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100.."
+METRICS = {
+    "c3": "routing instance-steps/sec (batched BR-0, 4096 instances, G=32, W=256)",
+    "c4": "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
+}
+WORKLOADS = {
+    "c3": "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100..",
+    "c4": "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000..",
+}
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -56,38 +67,38 @@ def kernel_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(workload: str, spl: int = 1):
-    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
-    profiles/traffic.json, or None if the kernel sources changed since that capture."""
+def _recorded(field: str, workload: str, spl: int):
     p = os.path.join(ROOT, "profiles", "traffic.json")
     try:
         rec = json.load(open(p))
         if rec.get("kernel_source_hash") == kernel_source_hash():
-            return rec["bytes_per_launch"].get(f"{workload}_spl{spl}")
+            return rec.get(field, {}).get(f"{workload}_spl{spl}")
     except Exception:
         pass
     return None
+
+
+def recorded_traffic(workload: str, spl: int = 1):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
+    profiles/traffic.json, or None if the kernel sources changed since that capture."""
+    return _recorded("bytes_per_launch", workload, spl)
 
 
 def recorded_instructions(workload: str, spl: int = 1):
     """Warp instructions per launch from the same ncu capture (None if the kernel changed)."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        rec = json.load(open(p))
-        if rec.get("kernel_source_hash") == kernel_source_hash():
-            return rec.get("warp_instructions_per_launch", {}).get(f"{workload}_spl{spl}")
-    except Exception:
-        pass
-    return None
+    return _recorded("warp_instructions_per_launch", workload, spl)
 
 
 def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
     """Bytes one instance-step has to move once: running-request state in, queue in,
-    assignments out, per-worker state in and out, slot edits."""
+    assignments out, per-worker state in and out, slot edits; for BR-H the prediction state
+    (4 bytes per slot read, 4 / Delta_T written) and the classifier rows of the refreshed
+    requests.  The library stores the prediction state in 5 bytes per slot (fp32 c_hat plus a
+    one-byte refresh stamp); the extra byte is layout cost and is not counted here."""
     A, G, W, H = cfg.G * cfg.B, cfg.G, cfg.W, cfg.H
     b = 4.0 * A + 8.0 * W + 4.0 * W + 20.0 * G + 28.0 * G + 24.0 + 8.0 * edits_per_step
     if H > 0:
-        b += 5.0 * A + 4.0 * H * A * rho + 5.0 * A / cfg.delta_T
+        b += 4.0 * A + 4.0 * H * A * rho + 4.0 * A / cfg.delta_T
     return b
 
 
@@ -125,6 +136,7 @@ class ClockSampler:
             rows = [r for r in rows if len(r) >= 9]
             if t0 is not None:
                 import datetime
+
                 def ts(r):
                     return datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
                 inside = [r for r in rows if t0 <= ts(r) <= t1]
@@ -178,53 +190,109 @@ def dist_setup(args):
     return world, rank, local, None
 
 
+def steps_per_launch_for(cfg, asked: int) -> int:
+    """Decode steps per br_step call: what was asked for, bounded by the configuration's length."""
+    return max(1, min(asked, cfg.steps))
+
+
 # ----------------------------------------------------------------------------- CPU arm
-def oracle_rate(cfg_name: str, budget_s: float, n_inst: int, max_steps: int):
-    """Instance-steps/s of the CPU checker, single thread, on the first n_inst instances."""
+def _oracle_worker(job):
+    """Runs the CPU checker on instances [first, first + n) of a configuration for at most
+    `budget_s` seconds or `max_steps` decode steps (a top-level function: pool workers are
+    started with `spawn`)."""
+    cfg_name, first, n, max_steps, budget_s = job
     import oracle
     cfg = wlm.get_config(cfg_name)
-    wl = wlm.make_workload(cfg, n_instances=n_inst)
-    orcs = [oracle.instance_from_workload(wl, i) for i in range(n_inst)]
-    probs = [wlm.term_probs_np(wl, k) for k in range(min(max_steps, 8))] if cfg.H > 0 else None
+    wl = wlm.make_workload(cfg, n_instances=n, first_instance=first)
+    orcs = [oracle.instance_from_workload(wl, i) for i in range(n)]
+    probs = [wlm.term_probs_np(wl, k) for k in range(min(max_steps, 4))] if cfg.H > 0 else None
     done = 0
     t0 = time.perf_counter()
     for k in range(max_steps):
         for i, o in enumerate(orcs):
             o.step(None if probs is None else probs[k % len(probs)][i])
-        done += n_inst
+        done += n
         if time.perf_counter() - t0 > budget_s:
             break
-    dt = time.perf_counter() - t0
+    return done, time.perf_counter() - t0
+
+
+def oracle_rate(cfg_name: str, budget_s: float, n_inst: int, max_steps: int):
+    """Instance-steps/s of the CPU checker, single thread, on the first n_inst instances."""
+    done, dt = _oracle_worker((cfg_name, 0, n_inst, max_steps, budget_s))
     return done / dt, done, dt
 
 
+def oracle_rate_all_cores(cfg_name: str, budget_s: float, n_per_proc: int, max_steps: int):
+    """Aggregate instance-steps/s of the checker with one process per host core, each on its own
+    instances.  The pool is started with `spawn` (a fork after CUDA initialisation can hang)."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0))
+    jobs = [(cfg_name, p * n_per_proc, n_per_proc, max_steps, budget_s) for p in range(cores)]
+    with mp.get_context("spawn").Pool(cores) as pool:
+        t0 = time.perf_counter()
+        res = pool.map(_oracle_worker, jobs)
+        wall = time.perf_counter() - t0
+    done = sum(r[0] for r in res)
+    rate = sum(r[0] / r[1] for r in res)
+    return rate, done, wall, cores
+
+
+def cpu_baselines(args):
+    """The checker as it stands on the host cores: the headline workload on one thread and on all
+    cores, and the other configurations on one thread, each on a bounded sample."""
+    out = {}
+    rate, done, dt = oracle_rate("c3", 12.0, 512, 500)
+    out["c3"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                 "sample": f"{done} instance-steps of c3 (first 512 instances, steps 0..{done // 512 - 1}), "
+                           f"{dt:.1f} s, single thread"}
+    try:
+        rate, done, wall, cores = oracle_rate_all_cores("c3", 6.0, 64, 500)
+        out["c3_all_cores"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": f"{done} instance-steps of c3, {cores} processes x 64 instances, "
+                                         f"{wall:.1f} s wall including process start"}
+    except Exception as ex:
+        out["c3_all_cores"] = {"error": repr(ex)}
+    for name, n, steps, budget in (("c4", 32, 100, 4.0), ("c1", 32, 2000, 3.0), ("c2", 32, 2000, 3.0)):
+        rate, done, dt = oracle_rate(name, budget, n, steps)
+        out[name] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                     "ms_per_instance_step": 1e3 / rate,
+                     "sample": f"{done} instance-steps of {name} ({n} instance(s)), {dt:.1f} s, single thread"}
+    return out
+
+
 def run_reference(args):
-    """The CPU checker as it stands, timed on host cores (rank 0 only)."""
+    """The CPU checker as it stands, timed on host cores (rank 0 only).  One step is the same
+    unit as on the GPU arm (--steps-per-launch decode steps of the batch), carried out on a
+    bounded sample of the batch: its first 32 instances."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
     cfg = wlm.get_config("c3")
     n_inst = 32
+    spl = steps_per_launch_for(cfg, args.steps_per_launch)
+    steps = min(args.steps, max(1, (cfg.steps - spl * args.warmup) // spl))
     wl = wlm.make_workload(cfg, n_instances=n_inst)
     orcs = [oracle.instance_from_workload(wl, i) for i in range(n_inst)]
-    for _ in range(args.warmup):
+    for _ in range(args.warmup * spl):
         for o in orcs:
             o.step()
     t0 = time.perf_counter()
-    for _ in range(args.steps):
+    for _ in range(steps * spl):
         for o in orcs:
             o.step()
     dt = time.perf_counter() - t0
-    val = n_inst * args.steps / dt
+    val = n_inst * steps * spl / dt
     line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "impl": "reference", "metric": METRICS["c3"], "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
-        "config": {"workload": C3_WORKLOAD, "sample": "the first 32 instances, one decode step of each per step"},
+        "config": {"workload": WORKLOADS["c3"], "steps_per_launch": spl,
+                   "sample": f"the first {n_inst} instances, {spl} decode steps of each per step"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"{n_inst} instances x {args.steps} steps of c3, single thread"},
+                         "sample": f"{n_inst} instances x {steps * spl} decode steps of c3, single thread"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -233,10 +301,11 @@ def run_reference(args):
 # ----------------------------------------------------------------------------- GPU arm
 class RotatingSets:
     """R independent instance sets of one configuration, stepped in rotation; one call of
-    step() is one launch that advances one set by `spl` decode steps."""
+    step() is one launch that advances one set by `spl` decode steps.  reset() puts every set
+    back to its initial snapshot (device copies), so that repeats time the same work."""
 
     def __init__(self, cfg_name, n_inst, n_sets, device, seed_offset=0, threads=0, probs_ring=1, spl=1,
-                 **params):
+                 start_steps=None, **params):
         import torch
         from paper_2605_06113_b200.binding import Router
         self.torch = torch
@@ -247,6 +316,7 @@ class RotatingSets:
             wl = wlm.make_workload(self.cfg, n_instances=n_inst, first_instance=seed_offset + r * n_inst)
             router = Router(wl, device=device, threads=threads, **params)
             st = router.device_state()
+            st0 = {k: v.clone() for k, v in st.items()}
             out = router.outputs(n_inst, n_steps=spl)
             probs = []
             if self.cfg.H > 0:
@@ -256,14 +326,32 @@ class RotatingSets:
                     probs.append(torch.stack([wlm.term_probs_torch(wl, j * spl + i, device, seeds_t=seeds_t, tab_t=tab_t)
                                               for i in range(spl)]).contiguous())
             calls = [router.prepare(st, out, pr, N=n_inst, first=0, n_steps=spl) for pr in (probs or [None])]
-            self.sets.append(dict(wl=wl, router=router, st=st, out=out, probs=probs, calls=calls))
+            self.sets.append(dict(wl=wl, router=router, st=st, st0=st0, out=out, probs=probs, calls=calls))
         self.router = self.sets[0]["router"]
         self.launch = 0
+        # Sets may start at different points of the configuration's trajectory (untimed launches
+        # bring them there); the snapshot that reset() restores is taken afterwards.
+        self.start_steps = [0] * n_sets
+        if start_steps is not None:
+            for j, s in enumerate(self.sets):
+                n = int(start_steps[j]) // spl
+                for i in range(n):
+                    s["calls"][i % len(s["calls"])]()
+                self.start_steps[j] = n * spl
+            torch.cuda.synchronize()
+            for s in self.sets:
+                s["st0"] = {k: v.clone() for k, v in s["st"].items()}
 
     def step(self):
         s = self.sets[self.launch % self.n_sets]
         s["calls"][(self.launch // self.n_sets) % len(s["calls"])]()
         self.launch += 1
+
+    def reset(self):
+        for s in self.sets:
+            for k, v in s["st"].items():
+                v.copy_(s["st0"][k])
+        self.launch = 0
 
     def counters_mean(self):
         t = self.torch
@@ -278,9 +366,9 @@ class RotatingSets:
         self.sets = []
 
 
-def time_launches(torch, fn, warmup, steps, dist=None):
-    for _ in range(warmup):
-        fn()
+def time_region(torch, fn, steps, dist=None):
+    """Device time of exactly `steps` calls of fn, bracketed by a barrier and a device
+    synchronisation on both sides; the slowest rank's time."""
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -298,6 +386,234 @@ def time_launches(torch, fn, warmup, steps, dist=None):
         dist.barrier()
         torch.cuda.synchronize()
     return ms
+
+
+def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, threads=0,
+                    seed_offset=0, dist=None, sampler=None, probs_ring=2):
+    """Times `launches` br_step calls of the batched configuration `wname`, `spl` decode steps per
+    call, `repeats` times.  Enough instance sets rotate that the data between two visits of a set
+    exceeds L2 and that no instance runs past the configuration's length.  The work of a decode
+    step changes along a configuration's trajectory (c3 starts with half-empty workers and a full
+    queue, so its first ~80 steps admit several times more requests than the rest), so the sets
+    start at evenly spaced points of the trajectory and the timed region is a stratified sample of
+    it (the whole of it when launches * spl reaches sets * configuration length).  Before every
+    repeat the sets return to their starting snapshots and one untimed call per set runs;
+    `warmup` untimed calls precede the first repeat."""
+    cfg = wlm.get_config(wname)
+    N = cfg.N
+    per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
+    n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
+    n_sets = max(n_sets, int(np.ceil((launches + n_sets) * spl / cfg.steps)))
+    prime = n_sets
+    per_set = -(-(launches + prime) // n_sets)                # launches a set sees in one repeat
+    span = per_set * spl
+    room = max(0, cfg.steps - span)
+    starts = [int(j * room / max(1, n_sets - 1)) // spl * spl for j in range(n_sets)]
+    sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
+                        probs_ring=probs_ring, spl=spl, start_steps=starts)
+    starts = list(sets.start_steps)
+    for _ in range(warmup):
+        sets.step()
+    torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.start()
+        time.sleep(0.3)                      # let the sampler come up before the timed regions
+    t0 = time.time()
+    reps = []
+    for _ in range(repeats):
+        sets.reset()
+        for _ in range(prime):
+            sets.step()
+        reps.append(time_region(torch, sets.step, launches, dist))
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
+    cnt = sets.counters_mean()
+    bad = sets.bad_status()
+    tpi = sets.router.params.threads
+    sets.close()
+    del sets
+    torch.cuda.empty_cache()
+    ms = float(np.median(reps))
+    # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
+    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
+    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
+    us_per_launch = 1e3 * ms / launches
+    return dict(ms=ms, ms_per_launch=ms / launches, us_per_launch=us_per_launch, n_sets=n_sets, N=N, spl=spl,
+                trajectory=f"sets start at decode steps {starts} of {cfg.steps} and advance {span} steps per repeat",
+                repeats_ms=[float(x) for x in reps], abytes_per_launch=abytes,
+                achieved=abytes / (us_per_launch * 1e-6) / 1e9, bad=bad, clocks=clocks, threads=tpi,
+                launches=launches, value=N * spl * launches / (ms * 1e-3))
+
+
+def kernel_name(wname):
+    return "br_small_kernel<2,4>" if wname == "c3" else "br_step_kernel<true,8,2,1>"
+
+
+def roofline_of(m, wname, peak, peak_kind, clocks=None):
+    """HBM roofline entry of one measurement.  `achieved` is the algorithmic bytes of a launch over
+    its measured duration (a normalised throughput: the kernel may move fewer bytes than that --
+    BR-0 advances loads without streaming the per-request state -- or more); `dram` is the DRAM
+    traffic ncu counted for the same launch shape over the same duration, i.e. the share of the
+    HBM bandwidth the kernel really uses; `issue` is what binds the step kernels."""
+    spl = m["spl"]
+    traffic = recorded_traffic(wname, spl)
+    r = {"bound": "hbm", "achieved": m["achieved"], "peak": peak, "unit": "GB/s",
+         "frac": m["achieved"] / peak, "frac_of_nominal_8TBs": m["achieved"] / NOMINAL_HBM_GBS,
+         "peak_kind": peak_kind, "traffic": traffic,
+         "achieved_kind": "algorithmic bytes per launch / measured launch time",
+         "algorithmic_bytes_per_launch": m["abytes_per_launch"],
+         "us_per_launch": m["us_per_launch"], "kernel": kernel_name(wname)}
+    if traffic:
+        dram = traffic / (m["us_per_launch"] * 1e-6) / 1e9
+        r["dram"] = {"achieved": dram, "unit": "GB/s", "frac": dram / peak,
+                     "traffic_over_algorithmic": traffic / m["abytes_per_launch"]}
+    winst = recorded_instructions(wname, spl)
+    if winst:
+        # what binds the step: instruction issue.  Peak = 148 SMs x 4 schedulers x 1 warp
+        # instruction per clock at the SM clock sampled during the run.
+        clk = ((clocks or {}).get("sm_mhz") or 1965.0) * 1e6
+        peak_issue = 148 * 4 * clk
+        ach = winst / (m["us_per_launch"] * 1e-6)
+        r["issue"] = {"bound": "alu", "achieved": ach / 1e9, "peak": peak_issue / 1e9,
+                      "unit": "G warp-instructions/s", "frac": ach / peak_issue,
+                      "warp_instructions_per_launch": winst}
+    return r
+
+
+def brief(m, roof):
+    return {"us_per_launch": round(m["us_per_launch"], 2), "us_per_decode_step": round(m["us_per_launch"] / m["spl"], 2),
+            "inst_steps_per_s": round(m["value"]), "frac": round(roof["frac"], 4),
+            "dram_frac": round(roof["dram"]["frac"], 4) if "dram" in roof else None,
+            "traffic_over_algorithmic": round(roof["dram"]["traffic_over_algorithmic"], 3) if "dram" in roof else None}
+
+
+def run_ours(args):
+    import torch
+    world, rank, local, dist = dist_setup(args)
+    device = f"cuda:{local}"
+    torch.cuda.set_device(local)
+    peak, peak_kind = measured_peaks()
+
+    # ---------------- headline: batched, several decode steps per launch ----------------
+    wname = args.workload
+    cfg = wlm.get_config(wname)
+    spl = steps_per_launch_for(cfg, args.steps_per_launch)
+    first, _ = shard_of(rank, world, cfg.N, 64)
+    m = measure_batched(torch, wname, device, args.steps, args.warmup, spl, repeats=args.repeats,
+                        threads=args.threads, seed_offset=first, dist=dist, sampler=ClockSampler(local))
+    N = m["N"]
+    value = world * m["value"]
+    clocks = m["clocks"]
+    roofline = roofline_of(m, wname, peak, peak_kind, clocks)
+    line = {
+        "metric": METRICS[wname], "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": m["ms_per_launch"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None,
+        # arithmetic of the path: Eq. 1 scores, loads and keys in 32-bit integers (ranges proven at
+        # br_create), 64-bit outputs; the BR-H workload scores Eq. 2 in fp64
+        "dtype": "int32" if wname == "c3" else "f64", "data": "synthetic",
+        "config": {"workload": WORKLOADS[wname],
+                   "step": f"one br_step call = one launch advancing {N} instances by {spl} decode steps "
+                           f"({N * spl} instance-steps)",
+                   "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
+                   "repeats": args.repeats,
+                   "timing": f"median of {args.repeats} repeats of the {args.steps}-call region (CUDA events; "
+                             f"before each repeat the sets return to their starting snapshots and one untimed "
+                             f"call per set runs)",
+                   "trajectory": m["trajectory"],
+                   "l2": f"{m['n_sets']} instance sets stepped in rotation: data touched between two visits of a "
+                         f"set exceeds the 126 MB L2; no instance runs past the configuration's {cfg.steps} steps",
+                   "threads_per_instance": m["threads"]},
+        "ms_per_step_min": min(m["repeats_ms"]) / args.steps, "ms_per_step_max": max(m["repeats_ms"]) / args.steps,
+        "roofline": roofline, "clocks": clocks, "gpu_launches": m["launches"],
+        "bad_status_instances": m["bad"],
+    }
+    summary = {f"{wname}_{spl}_steps_per_launch": brief(m, roofline)}
+
+    if rank == 0 and world == 1 and not args.quick and wname == "c3":
+        # the same workload with one decode step per launch (the form the latency path replays)
+        m1 = measure_batched(torch, wname, device, 400, 40, 1, repeats=5, threads=args.threads)
+        r1 = roofline_of(m1, wname, peak, peak_kind, clocks)
+        line["single_step_launches"] = {"value": m1["value"], "unit": UNIT, "ms_per_step": m1["ms_per_launch"],
+                                        "roofline": r1, "gpu_launches": m1["launches"], "repeats_ms": m1["repeats_ms"]}
+        summary["c3_1_step_per_launch"] = brief(m1, r1)
+        # ---------------- end to end through the host-buffer entry point ----------------
+        line["e2e"] = e2e_host(torch, device, args)
+        summary["e2e_c3_host_buffers"] = {"inst_steps_per_s": round(line["e2e"]["value"]),
+                                          "ms_per_step": round(line["e2e"]["ms_per_step"], 3)}
+        # ---------------- extras: c4 batched BR-H, stand-alone entry points, latency path ----------------
+        try:
+            line["extra"] = extras(torch, device, args, peak, peak_kind, summary)
+        except Exception as ex:  # keep the headline line even if an extra fails
+            line["extra"] = {"error": repr(ex)}
+        # ---------------- CPU baseline: the checker on host cores ----------------
+        try:
+            cb = cpu_baselines(args)
+            line["cpu_baseline"] = cb["c3"]
+            line["cpu_baseline_other"] = {k: v for k, v in cb.items() if k != "c3"}
+            summary["cpu_oracle_inst_steps_per_s"] = {k: (round(v["value"]) if "value" in v else None, v.get("cores"))
+                                                      for k, v in cb.items()}
+        except Exception as ex:
+            line["cpu_baseline"] = {"error": repr(ex)}
+    elif rank == 0:
+        line["e2e"] = None
+    line["summary"] = summary                 # last key: the tail of the line holds every headline figure
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def e2e_host(torch, device, args):
+    from paper_2605_06113_b200.binding import Router
+    cfg = wlm.get_config("c3")
+    wl = wlm.make_workload(cfg, n_instances=cfg.N, first_instance=1 << 20)
+    r = Router(wl, device=device, threads=args.threads)
+    st = {k: torch.from_numpy(np.ascontiguousarray(v).view(
+        {np.dtype(np.uint64): np.int64, np.dtype(np.uint32): np.int32}.get(v.dtype, v.dtype))).pin_memory()
+          for k, v in wl.state.items()}
+    out = {k: v.pin_memory() for k, v in r.outputs(cfg.N, device="cpu").items()}
+    steps = 30
+    up = down = 0
+    for _ in range(3):
+        r.step_host(st, out)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        up, down = r.step_host(st, out)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    r.close()
+    return {"value": cfg.N * steps / dt, "unit": UNIT, "h2d_bytes_per_step": up,
+            "d2h_bytes_per_step": down, "steps": steps, "ms_per_step": 1e3 * dt / steps,
+            "step": "one decode step of 4096 instances through br_step_host: pinned host snapshot up, "
+                    "kernel, snapshot and results down"}
+
+
+def extras(torch, device, args, peak, peak_kind, summary):
+    ex = {}
+    # c4: BR-H batched (H = 8), 4 decode steps per launch and one step per launch
+    for spl in (4, 1):
+        m = measure_batched(torch, "c4", device, 200 // spl, 20, spl, repeats=5)
+        roof = roofline_of(m, "c4", peak, peak_kind)
+        key = "c4_batched" if spl == 4 else "c4_single_step_launches"
+        ex[key] = {"value": m["value"], "unit": UNIT, "ms_per_step": m["ms_per_launch"], "steps_per_launch": spl,
+                   "repeats_ms": m["repeats_ms"], "roofline": roof}
+        summary[f"c4_{spl}_step{'s' if spl > 1 else ''}_per_launch"] = brief(m, roof)
+    # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
+    try:
+        ex["entry_points"] = entry_points(torch, device, peak)
+        summary["br_fscore_eq1_frac"] = round(ex["entry_points"]["br_fscore_eq1"]["roofline"]["frac"], 3)
+    except Exception as e:
+        ex["entry_points"] = {"error": repr(e)}
+    # latency path: one instance, one graph-replayed step per decode step
+    lat = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
+           latency_path(torch, "c4", device, 1000)]
+    ex["latency"] = lat
+    summary["latency_device_p50_us"] = {f"{l['workload']}(G={l['G']},W={l['W']},H={l['H']})": round(l["device_p50_us"], 1)
+                                        for l in lat}
+    summary["latency_host_p50_us"] = {l["workload"]: round(l["host_p50_us"], 1) for l in lat}
+    return ex
 
 
 def latency_path(torch, cfg_name, device, steps, overrides=None):
@@ -354,170 +670,6 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
             "phase_note": "phase split taken with the kernel's cycle counters on br_step_kernel (the "
                           "kernel that offers them); the latencies above are those of the kernel the "
                           "library picks for the shape"}
-
-
-def measure_batched(torch, wname, device, steps, warmup, spl, threads=0, seed_offset=0, dist=None,
-                    sampler=None, probs_ring=2, min_sets=0):
-    """Times `steps` decode steps of the batched configuration `wname`, `spl` steps per launch, on
-    enough rotating instance sets that no instance runs past the configuration's length."""
-    cfg = wlm.get_config(wname)
-    N = cfg.N
-    per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
-    n_sets = max(2, min_sets, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))),
-                 int(np.ceil((steps + warmup) / cfg.steps)))
-    sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
-                        probs_ring=probs_ring, spl=spl)
-    if sampler is not None:
-        sampler.start()
-        time.sleep(0.4)                      # let the sampler come up before the timed region
-    t0 = time.time()
-    ms = time_launches(torch, sets.step, -(-warmup // spl), steps // spl, dist)
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1) if sampler is not None else None
-    cnt = sets.counters_mean()
-    bad = sets.bad_status()
-    tpi = sets.router.params.threads
-    sets.close()
-    del sets
-    torch.cuda.empty_cache()
-    # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
-    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
-    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
-    us_per_launch = 1e3 * ms / (steps // spl)
-    return dict(ms=ms, ms_per_step=ms / steps, us_per_launch=us_per_launch, n_sets=n_sets, N=N,
-                abytes_per_launch=abytes, achieved=abytes / (us_per_launch * 1e-6) / 1e9, bad=bad,
-                clocks=clocks, threads=tpi, launches=steps // spl)
-
-
-def kernel_name(wname):
-    return "br_small_kernel<2,4>" if wname == "c3" else "br_step_kernel<true,8,2,1>"
-
-
-def run_ours(args):
-    import torch
-    world, rank, local, dist = dist_setup(args)
-    device = f"cuda:{local}"
-    torch.cuda.set_device(local)
-    peak, peak_kind = measured_peaks()
-
-    # ---------------- headline: batched, several decode steps per launch ----------------
-    wname = args.workload
-    cfg = wlm.get_config(wname)
-    spl = args.steps_per_launch if args.steps % args.steps_per_launch == 0 else 1
-    first, _ = shard_of(rank, world, cfg.N, 64)
-    m = measure_batched(torch, wname, device, args.steps, args.warmup, spl, threads=args.threads,
-                        seed_offset=first, dist=dist, sampler=ClockSampler(local))
-    N = m["N"]
-    value = world * N * args.steps / (m["ms"] * 1e-3)
-    roofline = {"bound": "hbm", "achieved": m["achieved"], "peak": peak, "unit": "GB/s",
-                "frac": m["achieved"] / peak, "frac_of_nominal_8TBs": m["achieved"] / NOMINAL_HBM_GBS,
-                "peak_kind": peak_kind, "traffic": recorded_traffic(wname, spl),
-                "algorithmic_bytes_per_launch": m["abytes_per_launch"],
-                "us_per_launch": m["us_per_launch"], "kernel": kernel_name(wname)}
-    winst = recorded_instructions(wname, spl)
-    clocks = m["clocks"]
-    if winst:
-        # what actually binds the step: instruction issue.  Peak = 148 SMs x 4 schedulers x 1 warp
-        # instruction per clock at the SM clock sampled during the run.
-        clk = (clocks.get("sm_mhz") or 1965.0) * 1e6
-        peak_issue = 148 * 4 * clk
-        ach = winst / (m["us_per_launch"] * 1e-6)
-        roofline["issue"] = {"bound": "alu", "achieved": ach / 1e9, "peak": peak_issue / 1e9,
-                             "unit": "G warp-instructions/s", "frac": ach / peak_issue,
-                             "warp_instructions_per_launch": winst}
-    line = {
-        "metric": METRIC if wname == "c3" else "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
-        "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None,
-        # arithmetic of the path: Eq. 1 scores, loads and keys in 32-bit integers (ranges proven at
-        # br_create), 64-bit outputs; the BR-H workload scores Eq. 2 in fp64
-        "dtype": "int32" if wname == "c3" else "f64", "data": "synthetic",
-        "config": {"workload": (C3_WORKLOAD if wname == "c3"
-                                else "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000.."),
-                   "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
-                   "l2": f"{m['n_sets']} instance sets stepped in rotation ({spl} decode steps per launch and "
-                         f"set): data touched between two visits of a set exceeds the 126 MB L2; no instance "
-                         f"runs past the configuration's {cfg.steps} steps",
-                   "threads_per_instance": m["threads"]},
-        "roofline": roofline, "clocks": clocks, "gpu_launches": m["launches"],
-        "bad_status_instances": m["bad"],
-    }
-
-    if rank == 0 and world == 1 and not args.quick and wname == "c3":
-        # the same workload with one decode step per launch (the form the latency path replays)
-        m1 = measure_batched(torch, wname, device, 1920, 80, 1, threads=args.threads)
-        line["single_step_launches"] = {
-            "value": N * 1920 / (m1["ms"] * 1e-3), "unit": UNIT, "ms_per_step": m1["ms_per_step"],
-            "roofline": {"bound": "hbm", "achieved": m1["achieved"], "peak": peak, "unit": "GB/s",
-                         "frac": m1["achieved"] / peak, "traffic": recorded_traffic(wname, 1),
-                         "algorithmic_bytes_per_launch": m1["abytes_per_launch"]},
-            "gpu_launches": 1920}
-        # ---------------- end to end through the host-buffer entry point ----------------
-        line["e2e"] = e2e_host(torch, device, args)
-        # ---------------- extras: c4 batched BR-H, latency path ----------------
-        try:
-            line["extra"] = extras(torch, device, args, peak)
-        except Exception as ex:  # keep the headline line even if an extra fails
-            line["extra"] = {"error": repr(ex)}
-        # ---------------- CPU baseline: the checker on host cores ----------------
-        rate, done, dt = oracle_rate("c3", 20.0, 1024, 500)
-        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{done} instance-steps of c3 (first 1024 instances, steps 0..{done // 1024 - 1}), "
-                                          f"{dt:.1f} s, single thread"}
-    elif rank == 0:
-        line["e2e"] = None
-    if rank == 0:
-        print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
-
-
-def e2e_host(torch, device, args):
-    from paper_2605_06113_b200.binding import Router
-    cfg = wlm.get_config("c3")
-    wl = wlm.make_workload(cfg, n_instances=cfg.N, first_instance=1 << 20)
-    r = Router(wl, device=device, threads=args.threads)
-    st = {k: torch.from_numpy(np.ascontiguousarray(v).view(
-        {np.dtype(np.uint64): np.int64, np.dtype(np.uint32): np.int32}.get(v.dtype, v.dtype))).pin_memory()
-          for k, v in wl.state.items()}
-    out = {k: v.pin_memory() for k, v in r.outputs(cfg.N, device="cpu").items()}
-    steps = 30
-    up = down = 0
-    for _ in range(3):
-        r.step_host(st, out)
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        up, down = r.step_host(st, out)
-    torch.cuda.synchronize()
-    dt = time.perf_counter() - t0
-    r.close()
-    return {"value": cfg.N * steps / dt, "unit": UNIT, "h2d_bytes_per_step": up,
-            "d2h_bytes_per_step": down, "steps": steps, "ms_per_step": 1e3 * dt / steps}
-
-
-def extras(torch, device, args, peak):
-    ex = {}
-    # c4: BR-H batched (H = 8), 4 decode steps per launch and one step per launch
-    for spl in (4, 1):
-        m = measure_batched(torch, "c4", device, 400, 40, spl)
-        ex["c4_batched" if spl == 4 else "c4_single_step_launches"] = {
-            "value": m["N"] * 400 / (m["ms"] * 1e-3), "unit": UNIT, "ms_per_step": m["ms_per_step"],
-            "steps_per_launch": spl,
-            "roofline": {"bound": "hbm", "achieved": m["achieved"], "peak": peak, "unit": "GB/s",
-                         "frac": m["achieved"] / peak, "traffic": recorded_traffic("c4", spl),
-                         "algorithmic_bytes_per_launch": m["abytes_per_launch"],
-                         "kernel": kernel_name("c4")}}
-    # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
-    try:
-        ex["entry_points"] = entry_points(torch, device, peak)
-    except Exception as e:
-        ex["entry_points"] = {"error": repr(e)}
-    # latency path: one instance, one graph-replayed step per decode step
-    ex["latency"] = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
-                     latency_path(torch, "c4", device, 1000)]
-    return ex
 
 
 def _time_call(torch, fn, reps=20, warm=3):
@@ -606,10 +758,11 @@ def entry_points(torch, device, peak):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3840)
-    ap.add_argument("--warmup", type=int, default=160)
+    ap.add_argument("--steps", type=int, default=60, help="br_step calls in the timed region")
+    ap.add_argument("--warmup", type=int, default=10, help="untimed br_step calls before the first repeat")
     ap.add_argument("--steps-per-launch", type=int, default=16,
-                    help="decode steps advanced by one launch (one br_step call with n_steps); used when it divides --steps")
+                    help="decode steps advanced by one br_step call (batch.n_steps)")
+    ap.add_argument("--repeats", type=int, default=7, help="repeats of the timed region; the median is reported")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="headline measurement only")
@@ -617,8 +770,9 @@ def main():
                     help="batched configuration timed as the headline (c4 is used for profiling the BR-H kernel)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.repeats = max(args.repeats, 1)
     if args.impl == "reference":
-        args.steps = min(args.steps, 400)
+        args.steps = min(args.steps, 25)
         run_reference(args)
     else:
         run_ours(args)
