@@ -91,3 +91,61 @@ def run_parity(cfg, n_inst, steps, threads=0, fscore=False, launch_steps=1, firs
                 compare_state(cfg, st_np, o, i, k)
     r.close()
     return np.array(traces)
+
+
+# ---- whole batches: the checker fanned out over host processes -------------------------------
+def oracle_chunk(job):
+    """Runs the checker on instances [first, first + n) of a configuration for `steps` decode
+    steps.  Returns the per-step outputs (assign as int16, load, trace, counters) and the final
+    snapshot of every instance.  Top-level so that a `spawn` pool can import it."""
+    name, overrides, first, n, steps = job
+    cfg = wlm.get_config(name, **overrides)
+    wl = wlm.make_workload(cfg, n_instances=n, first_instance=first)
+    orcs = [oracle.instance_from_workload(wl, i) for i in range(n)]
+    assign = np.empty((steps, n, cfg.W), dtype=np.int16)
+    load = np.empty((steps, n, cfg.G), dtype=np.int64)
+    trace = np.empty((steps, n, 3), dtype=np.int64)
+    cnt = np.empty((steps, n, 4), dtype=np.int64)
+    c_prev = [o.get_state()["counters"].copy() for o in orcs]
+    for k in range(steps):
+        probs = wlm.term_probs_np(wl, k) if cfg.H > 0 else None
+        for i, o in enumerate(orcs):
+            a, l, t, _ = o.step(None if probs is None else probs[i])
+            assign[k, i] = a; load[k, i] = l; trace[k, i] = t
+            c1 = o.get_state()["counters"].copy()
+            cnt[k, i] = (c1 - c_prev[i])[:4]
+            c_prev[i] = c1
+    fin = [o.get_state() for o in orcs]
+    return first, assign, load, trace, cnt, fin
+
+
+def oracle_batch(name, n_total, steps, overrides=None, chunk=None):
+    """The checker on instances 0..n_total-1, one process per host core (`spawn`: the parent has
+    CUDA initialised).  Returns the concatenated per-step outputs, the final snapshots and the
+    number of processes used."""
+    import multiprocessing as mp
+    import os
+    cores = len(os.sched_getaffinity(0))
+    chunk = chunk or max(1, -(-n_total // (cores * 2)))
+    jobs = [(name, overrides or {}, f, min(chunk, n_total - f), steps) for f in range(0, n_total, chunk)]
+    procs = min(cores, len(jobs))
+    if procs <= 1:
+        res = [oracle_chunk(j) for j in jobs]
+    else:
+        with mp.get_context("spawn").Pool(procs) as pool:
+            res = pool.map(oracle_chunk, jobs)
+    res.sort(key=lambda r: r[0])
+    assign = np.concatenate([r[1] for r in res], axis=1)
+    load = np.concatenate([r[2] for r in res], axis=1)
+    trace = np.concatenate([r[3] for r in res], axis=1)
+    cnt = np.concatenate([r[4] for r in res], axis=1)
+    fin = [s for r in res for s in r[5]]
+    return assign, load, trace, cnt, fin, procs
+
+
+def compare_state_dict(cfg, st_np, s, i, k):
+    """compare_state against a snapshot dictionary of the checker (as oracle_chunk returns it)."""
+    class _Snap:
+        def get_state(self_inner):
+            return s
+    compare_state(cfg, st_np, _Snap(), i, k)

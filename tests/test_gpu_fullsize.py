@@ -95,6 +95,7 @@ def test_c3_full_batch_sixteen_steps_per_launch():
         assert int((out["status"] & ~1).ne(0).sum()) == 0
         tr = out["trace"]; load = out["load"]
         assert torch.equal(tr[:, :, 0], load.max(2).values) and torch.equal(tr[:, :, 2], load.sum(2))
+        assert torch.equal(tr[:, :, 1], load.min(2).values)
         ah = out["assign"][:, idx].cpu().numpy(); lh = load[:, idx].cpu().numpy(); th = tr[:, idx].cpu().numpy()
         for j in range(S):
             for c, i in enumerate(idx):
@@ -132,6 +133,7 @@ def test_c4_full_batch_four_steps_per_launch():
         assert int((out["status"] & ~1).ne(0).sum()) == 0
         tr = out["trace"]; load = out["load"]
         assert torch.equal(tr[:, :, 0], load.max(2).values) and torch.equal(tr[:, :, 2], load.sum(2))
+        assert torch.equal(tr[:, :, 1], load.min(2).values)
         ah = out["assign"][:, idx].cpu().numpy(); lh = load[:, idx].cpu().numpy(); th = tr[:, idx].cpu().numpy()
         for j in range(S):
             probs_np = wlm.term_probs_np(wl, launch * S + j, instances=idx)
