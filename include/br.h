@@ -41,7 +41,7 @@ extern "C" {
 
 /* compiled limits */
 #define BR_MAX_G      64
-#define BR_MAX_H      16
+#define BR_MAX_H      80     /* the lookahead the paper deploys (Section 5.1 "Our methods")   */
 #define BR_MAX_B     256     /* B must be a multiple of 8                     */
 #define BR_MAX_W    4096     /* W must be a multiple of 4                     */
 #define BR_MAX_RMAX    5     /* Stage 2 enumerates 2^R_max - 1 <= 31 subsets   */

@@ -210,6 +210,7 @@ class Instance:
     def set_state(self, k, next_id, act_base, act_id=None, chat=None, tau=None,
                   wq_s=None, wq_id=None, wq_n=0):
         A = self.G * self.B
+        assert 0 <= int(wq_n) <= self.W, "queue length beyond the capacity W"
         ab = np.ascontiguousarray(act_base, dtype=np.int32).reshape(A)
         ai = None if act_id is None else np.ascontiguousarray(act_id, dtype=np.uint32).reshape(A)
         ch = None if chat is None else np.ascontiguousarray(chat, dtype=np.float32).reshape(A)

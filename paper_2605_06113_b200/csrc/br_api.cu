@@ -64,7 +64,9 @@ step_kernel_t pick_kernel_gw(bool fp, int H, int lean)
     if (H == 0) return br::br_step_kernel<true, 0, GW, 0>;
     if (H <= 4) return lean ? br::br_step_kernel<true, 4, GW, 1> : br::br_step_kernel<true, 4, GW, 0>;
     if (H <= 8) return lean ? br::br_step_kernel<true, 8, GW, 1> : br::br_step_kernel<true, 8, GW, 0>;
-    return lean ? br::br_step_kernel<true, 16, GW, 1> : br::br_step_kernel<true, 16, GW, 0>;
+    if (H <= 16) return lean ? br::br_step_kernel<true, 16, GW, 1> : br::br_step_kernel<true, 16, GW, 0>;
+    // longer horizons (up to BR_MAX_H): projected loads and margins live in shared memory
+    return lean ? br::br_step_kernel<true, BR_MAX_H, GW, 1> : br::br_step_kernel<true, BR_MAX_H, GW, 0>;
 }
 
 step_kernel_t pick_kernel(bool fp, int H, int G, int lean)
@@ -162,6 +164,12 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     a.block_sync = (per_block > 1 && b->n_instances % per_block == 0) ? 1 : 0;
     a.smem_per_inst = (int32_t)ctx->smem;
     const int blocks = (b->n_instances + per_block - 1) / per_block;
+    if (ctx->smem * per_block > 48 * 1024) {
+        // beyond the default limit: opt the kernel in (br_create has checked the device maximum)
+        cudaError_t eo = cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)(ctx->smem * per_block));
+        if (eo != cudaSuccess) return cuda_fail(eo, "cudaFuncSetAttribute(shared memory)");
+    }
     cudaError_t e = launch_overlapped(kern, blocks, tpi * per_block, ctx->smem * per_block, stream, a, overlap);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
@@ -270,7 +278,9 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         // The single-request arg-max may use the concavity of Eq. 2 only if no segment slope
         // alpha D - beta sum_{h in P} d_h (P any set of passed kinks) is within rounding distance of
         // zero: then fp64 scores of integer lengths are strictly ordered on both sides of the peak.
-        {
+        // The 2^(H+1) slopes are enumerated for H <= 16; longer horizons score every request.
+        a.peak_ok = 0;
+        if (H <= 16) {
             const int n = H + 1;
             double min_abs = 1e300;
             for (unsigned mask = 0; mask < (1u << n); ++mask) {
@@ -286,6 +296,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G; a.peak_ok = 0;
     }
     ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
+    if (ctx->smem > 227 * 1024) { delete ctx; return BR_EINVAL; }      // one instance must fit a thread block's shared memory
     // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 512 waiting requests,
     // arrivals served by one Philox call, and negative queue keys scoring below every waiting request
     ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode != 2 &&
@@ -593,7 +604,8 @@ int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int
     const int tiles = (n_requests + br::kFsTile - 1) / br::kFsTile;
     dim3 grid(tiles, batch->n_instances);
     void (*kern)(const br::FscoreArgs) = ctx->H == 0 ? br::br_fscore_kernel<0> : ctx->H <= 4 ? br::br_fscore_kernel<4>
-                                       : ctx->H <= 8 ? br::br_fscore_kernel<8> : br::br_fscore_kernel<16>;
+                                       : ctx->H <= 8 ? br::br_fscore_kernel<8>
+                                       : ctx->H <= 16 ? br::br_fscore_kernel<16> : br::br_fscore_kernel<BR_MAX_H>;
     kern<<<grid, 256, 0, (cudaStream_t)batch->stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_fscore launch");

@@ -42,7 +42,8 @@ __device__ __forceinline__ long long fscore_key(const FscoreArgs &a, int delta, 
 // Thread t of a block owns worker g = t % G for the whole tile (its margins and discounts stay in
 // registers) and walks the requests slice, slice + n_slices, ...: thread t writes elements
 // t, t + n_slices * G, ... of the tile's [request][worker] rows, so every store instruction of a
-// warp covers consecutive addresses.  HM bounds H at compile time (loops over h unrolled).
+// warp covers consecutive addresses.  HM bounds H at compile time (loops over h unrolled); HM > 16
+// stands for any longer horizon: the margins are then read from shared memory in a plain loop.
 template <int HM>
 __global__ void __launch_bounds__(256) br_fscore_kernel(const FscoreArgs a)
 {
@@ -74,14 +75,17 @@ __global__ void __launch_bounds__(256) br_fscore_kernel(const FscoreArgs a)
     const int n_slices = blockDim.x / G;
     const int slice = tid / G, g = tid - slice * G;
     if (slice < n_slices) {
-        double md[HM + 1], dd[HM + 1];
+        constexpr bool LONG = HM > 16;
+        constexpr int HR = LONG ? 0 : HM;
+        double md[HR + 1], dd[HR + 1];
         long long m0 = m_s[g * H1], mmin = m0;
 #pragma unroll
-        for (int h = 0; h <= HM; ++h) {
+        for (int h = 0; h <= HR; ++h) {
             md[h] = h <= H ? (double)m_s[g * H1 + h] : 0.0;
             dd[h] = h <= H ? a.d[h] : 0.0;
             if (h <= H) mmin = min(mmin, m_s[g * H1 + h]);
         }
+        if (LONG) for (int h = 1; h <= H; ++h) mmin = min(mmin, m_s[g * H1 + h]);
         const long long Gl = (long long)G;
 #pragma unroll 4
         for (int i = slice; i < n; i += n_slices) {
@@ -94,9 +98,17 @@ __global__ void __launch_bounds__(256) br_fscore_kernel(const FscoreArgs a)
             } else {
                 const double dl = (double)si;
                 double pen = 0.0;
-                if ((long long)si > mmin) {                                 // else every (s - m_h)_+ is zero
+                if (LONG) {
+                    if ((long long)si > mmin) {
+                        for (int h = 0; h <= H; ++h) {
+                            double over = __dsub_rn(dl, (double)m_s[g * H1 + h]);
+                            over = over > 0.0 ? over : 0.0;
+                            pen = __dadd_rn(pen, __dmul_rn(a.d[h], over));
+                        }
+                    }
+                } else if ((long long)si > mmin) {                          // else every (s - m_h)_+ is zero
 #pragma unroll
-                    for (int h = 0; h <= HM; ++h) {
+                    for (int h = 0; h <= HR; ++h) {
                         if (h <= H) {
                             double over = __dsub_rn(dl, md[h]);
                             over = over > 0.0 ? over : 0.0;

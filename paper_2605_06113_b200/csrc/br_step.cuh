@@ -57,6 +57,7 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     n += 4 * (size_t)G * (H + 1) * 2;            // Lh_s, Ch_s (PREDICT buckets: load sums, counts)
     n += 4 * (size_t)G;                          // sub_load
     n += 8 * (size_t)G * occ_words;              // fin_w
+    n += 8 * (size_t)(H + 1) + 4 * (size_t)((H + 2) / 2 * 2);   // md_s (fp64 margins of the selected worker), M_s (envelope)
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
     if (H > 0) n += 2 * (size_t)G * B;           // refresh_list
     return (n + 15) & ~(size_t)15;
@@ -64,10 +65,13 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
 
 // Order- and sign-preserving key of a score: Eq. 1 in integers (FP = false) or Eq. 2 in
 // fp64 evaluated term by term in h (FP = true).
-template <bool FP, int HM>
+// SL: the horizon is too long for registers; the margins of the selected worker are read from
+// shared memory (mds) and the loops over h are not unrolled.
+template <bool FP, int HM, bool SL = false>
 struct Scorer {
     int mi;                 // Eq. 1 margin
-    double md[HM + 1];      // Eq. 2 margins
+    double md[SL ? 1 : HM + 1];   // Eq. 2 margins
+    const double *mds;      // Eq. 2 margins in shared memory (SL)
     int mmin;               // min_h m_{g,h}: at or below it the Eq. 2 penalty is exactly zero
 
     __device__ __forceinline__ long long key(const StepArgs &a, int delta) const
@@ -79,12 +83,21 @@ struct Scorer {
         } else {
             const double dl = (double)delta;
             double pen = 0.0;
-#pragma unroll
-            for (int h = 0; h <= HM; ++h) {
-                if (h <= a.H) {
-                    double over = __dsub_rn(dl, md[h]);     // exact: integers below 2^53
+            if (SL) {
+#pragma unroll 4
+                for (int h = 0; h <= a.H; ++h) {
+                    double over = __dsub_rn(dl, mds[h]);
                     over = over > 0.0 ? over : 0.0;
                     pen = __dadd_rn(pen, __dmul_rn(a.d[h], over));
+                }
+            } else {
+#pragma unroll
+                for (int h = 0; h <= HM; ++h) {
+                    if (h <= a.H) {
+                        double over = __dsub_rn(dl, md[h]);     // exact: integers below 2^53
+                        over = over > 0.0 ? over : 0.0;
+                        pen = __dadd_rn(pen, __dmul_rn(a.d[h], over));
+                    }
                 }
             }
             return key_of_double(__dsub_rn(__dmul_rn(a.aD, dl), __dmul_rn(a.beta, pen)));
@@ -163,6 +176,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     extern __shared__ __align__(16) unsigned char smem_all[];
     // a.tpi threads serve one instance; a block holds blockDim.x / a.tpi instances (more than one
     // only when tpi == 32, so that an instance-wide barrier is a warp barrier)
+    constexpr bool SL = HM > 16;          // long horizons: projected loads, envelope and margins in shared memory
+    constexpr int HR = SL ? 0 : HM;       // horizon offsets kept in registers
     const int NT = a.tpi;
     const int tid = threadIdx.x % NT, lane = tid & 31, warp = tid >> 5;
     const int in_block = threadIdx.x / NT, per_block = blockDim.x / NT;
@@ -188,7 +203,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_id + W);     // [G][OW]
     unsigned long long *end_mask = occ + (size_t)G * OW;                            // [G][OW]
     unsigned long long *fin_w = end_mask + (size_t)G * OW;                          // [G][OW] slots whose draw says "ends"
-    unsigned *Lh_s = reinterpret_cast<unsigned *>(fin_w + (size_t)G * OW);          // [G][H1]
+    double *md_s = reinterpret_cast<double *>(fin_w + (size_t)G * OW);              // [H1] margins of the selected worker
+    int *M_s = reinterpret_cast<int *>(md_s + H1);                                  // [H1 rounded up to even] envelope
+    unsigned *Lh_s = reinterpret_cast<unsigned *>(M_s + (H1 + 1) / 2 * 2);          // [G][H1]
     unsigned *Ch_s = Lh_s + (size_t)G * H1;                                         // [G][H1]
     unsigned *sub_load = Ch_s + (size_t)G * H1;                                     // [G]
     unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
@@ -245,16 +262,17 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 
     // router registers: lane owns workers lane and lane + 32
     int cap[GW];
-    int L[GW][HM + 1];
-    int Mh[HM + 1];
+    int L[GW][HR + 1];
+    int Mh[HR + 1];
+    int *const L_s = reinterpret_cast<int *>(Lh_s);     // SL: the buckets become L_g(k+h) in place
 #pragma unroll
-    for (int h = 0; h <= HM; ++h) Mh[h] = 0;
+    for (int h = 0; h <= HR; ++h) Mh[h] = 0;
 #pragma unroll
     for (int w = 0; w < GW; ++w) {
         const int g = lane + 32 * w;
         cap[w] = -1;
 #pragma unroll
-        for (int h = 0; h <= HM; ++h) L[w][h] = 0;
+        for (int h = 0; h <= HR; ++h) L[w][h] = 0;
         if (warp == 0 && g < G) {
             int na = g_nact[g];
             if (na < 0 || na > B) { prologue_status |= BR_ST_BAD_STATE; na = na < 0 ? 0 : B; }
@@ -415,10 +433,34 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             for (int e = tid; e < n_ref; e += NT) {
                 const int s0 = refresh_list[e];
                 const float *q = probs + (size_t)s0 * H;
-                float qv[HM > 0 ? HM : 1];
+                if (SL) {
+                    // long classifier rows stay in memory: one pass for p_fin, one for c*
+                    double surv = 1.0, cs = 0.0;
+                    for (int h = 0; h < H; ++h) {
+                        cs = __dadd_rn(cs, surv);
+                        surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
+                    }
+                    double v = (double)H;
+                    if (__dsub_rn(1.0, surv) >= (double)a.gate) {
+                        v = cs;
+                        if (v < (double)a.c_floor) v = (double)a.c_floor;
+                        if (v > (double)H) v = (double)H;
+                    }
+                    const float c = (float)v;
+                    const int cur = g_base[s0] + k;
+                    g_chat0[s0] = c;
+                    g_kref[s0] = (uint8_t)(k & 255);
+                    int nh = (int)floorf(c);
+                    nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                    const int g = (int)__umulhi((unsigned)s0, a.magic_B);
+                    atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
+                    atomicAdd(&Ch_s[g * H1 + nh], 1u);
+                    continue;
+                }
+                float qv[HR > 0 ? HR : 1];
                 if ((H & 3) == 0) {
 #pragma unroll
-                    for (int h = 0; h < HM; h += 4) {
+                    for (int h = 0; h < HR; h += 4) {
                         if (h < H) {
                             const float4 qq = *reinterpret_cast<const float4 *>(q + h);
                             qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
@@ -426,19 +468,19 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     }
                 } else {
 #pragma unroll
-                    for (int h = 0; h < HM; ++h) if (h < H) qv[h] = q[h];
+                    for (int h = 0; h < HR; ++h) if (h < H) qv[h] = q[h];
                 }
                 const int cur = g_base[s0] + k;
                 // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
                 // clearly below the gate the fp64 product cannot reach it and is not evaluated
                 float qsum = 0.0f, qmin = 0.0f;
 #pragma unroll
-                for (int h = 0; h < HM; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
+                for (int h = 0; h < HR; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
                 double p_fin = 0.0;
                 if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
                     double surv = 1.0;
 #pragma unroll
-                    for (int h = 0; h < HM; ++h)
+                    for (int h = 0; h < HR; ++h)
                         if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
                     p_fin = __dsub_rn(1.0, surv);
                 }
@@ -447,7 +489,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     // gate open: E[min(r, H)] = sum_h prod_{j<h} (1 - q_j), clipped to [floor, H]
                     double sv = 1.0, cs = 0.0;
 #pragma unroll
-                    for (int h = 0; h < HM; ++h) {
+                    for (int h = 0; h < HR; ++h) {
                         if (h < H) {
                             cs = __dadd_rn(cs, sv);
                             sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
@@ -472,27 +514,53 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 
         if (warp == 0) {
             // ================= ROUTE (warp 0 only, warp-synchronous) =================
-            if (H > 0) {
+            if (SL) {
+                // buckets -> L_g(k+h) in place (each lane owns the rows of its workers), then the envelope
+                // with the lanes spread over h
 #pragma unroll
                 for (int w = 0; w < GW; ++w) {
                     const int g = lane + 32 * w;
-                    int accT = 0, accC = 0;
-#pragma unroll
-                    for (int h = HM; h >= 0; --h) {
-                        if (g < G && h <= H) { accT += (int)Lh_s[g * H1 + h]; accC += (int)Ch_s[g * H1 + h]; }
-                        L[w][h] = (g < G && h <= H) ? accT + h * accC : 0;
+                    if (g < G) {
+                        int accT = 0, accC = 0;
+                        for (int h = H; h >= 0; --h) {
+                            accT += (int)Lh_s[g * H1 + h]; accC += (int)Ch_s[g * H1 + h];
+                            L_s[g * H1 + h] = accT + h * accC;
+                        }
+                        L[w][0] = accT;
                     }
                 }
-            }
+                __syncwarp();
+                for (int h = lane; h <= H; h += 32) {
+                    int v = L_s[h];
+                    for (int g = 1; g < G; ++g) v = max(v, L_s[g * H1 + h]);
+                    M_s[h] = v;
+                }
+                __syncwarp();
+                Mh[0] = M_s[0];
+            } else {
+                if (H > 0) {
 #pragma unroll
-            for (int h = 0; h <= HM; ++h) {
-                int v = L[0][h];
+                    for (int w = 0; w < GW; ++w) {
+                        const int g = lane + 32 * w;
+                        int accT = 0, accC = 0;
 #pragma unroll
-                for (int w = 1; w < GW; ++w) v = max(v, L[w][h]);
-                Mh[h] = (h <= H) ? __reduce_max_sync(kFull, v) : 0;
+                        for (int h = HR; h >= 0; --h) {
+                            if (g < G && h <= H) { accT += (int)Lh_s[g * H1 + h]; accC += (int)Ch_s[g * H1 + h]; }
+                            L[w][h] = (g < G && h <= H) ? accT + h * accC : 0;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h <= HR; ++h) {
+                    int v = L[0][h];
+#pragma unroll
+                    for (int w = 1; w < GW; ++w) v = max(v, L[w][h]);
+                    Mh[h] = (h <= H) ? __reduce_max_sync(kFull, v) : 0;
+                }
             }
 
-            Scorer<FP, HM> sc;
+            Scorer<FP, HM, SL> sc;
+            sc.mds = md_s;
             // margins of worker g -> every lane's scorer
             auto load_margins = [&](int g) {
                 const int src = g & 31;
@@ -502,10 +570,20 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 #pragma unroll
                     for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[0] - L[w][0];
                     sc.mi = __shfl_sync(kFull, mine, src);
+                } else if (SL) {
+                    int mmin = 0x7FFFFFFF;
+                    __syncwarp();                          // earlier readers of md_s are done
+                    for (int h = lane; h <= H; h += 32) {
+                        const int mh = M_s[h] - L_s[g * H1 + h];
+                        md_s[h] = (double)mh;
+                        mmin = min(mmin, mh);
+                    }
+                    sc.mmin = __reduce_min_sync(kFull, mmin);
+                    __syncwarp();
                 } else {
                     int mmin = 0x7FFFFFFF;
 #pragma unroll
-                    for (int h = 0; h <= HM; ++h) {
+                    for (int h = 0; h <= HR; ++h) {
                         int mine = Mh[h] - L[0][h];
 #pragma unroll
                         for (int w = 1; w < GW; ++w) if (set == w) mine = Mh[h] - L[w][h];
@@ -562,7 +640,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int src = warp_argmax_lane32(bk, (unsigned)bkey & posmask, wk);
                     const int res = __shfl_sync(kFull, bkey, src);
                     return res > 0 ? res : 0;
-                } else if (a.peak_ok) {
+                } else if (!SL && a.peak_ok) {
                     // Eq. 2 is concave and piecewise linear in s with kinks at the m_{g,h}: it rises up
                     // to s* = the smallest kink at which the slope alpha D - beta sum_{m_h <= kink} d_h
                     // is no longer positive, and falls after it.  br_create has checked that no such
@@ -572,10 +650,10 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     // evaluations of Eq. 2.
                     double mine = 0.0;
 #pragma unroll
-                    for (int h = 0; h <= HM; ++h) if (lane == h) mine = sc.md[h];
+                    for (int h = 0; h <= HR; ++h) if (lane == h) mine = sc.md[h];
                     double wsum = 0.0;
 #pragma unroll
-                    for (int h = 0; h <= HM; ++h) if (h <= H && sc.md[h] <= mine) wsum = __dadd_rn(wsum, a.d[h]);
+                    for (int h = 0; h <= HR; ++h) if (h <= H && sc.md[h] <= mine) wsum = __dadd_rn(wsum, a.d[h]);
                     const bool past = lane <= H && !(a.aD > __dmul_rn(a.beta, wsum));
                     const int sstar = (int)__reduce_min_sync(kFull, past ? (unsigned)(int)mine : 0x7FFFFFFFu);
                     const int thr = sstar >= (1 << (31 - WL)) ? 0x7FFFFFFF : ((sstar << WL) | (int)posmask);
@@ -658,14 +736,23 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         if (set == w) {
                             cap[w] -= 1;
 #pragma unroll
-                            for (int h = 0; h <= HM; ++h) if (h <= H) L[w][h] += s;
+                            for (int h = 0; h <= HR; ++h) if (h <= H) L[w][h] += s;
                         }
                     }
                 }
                 // envelope: only worker g grew, so M_h = max(M_h, L_g(k+h))
+                if (SL) {
+                    for (int h = lane; h <= H; h += 32) {
+                        const int v = L_s[g * H1 + h] + s;
+                        L_s[g * H1 + h] = v;
+                        M_s[h] = max(M_s[h], v);
+                    }
+                    __syncwarp();
+                    Mh[0] = M_s[0];
+                }
 #pragma unroll
-                for (int h = 0; h <= HM; ++h) {
-                    if (h <= H) {
+                for (int h = 0; h <= HR; ++h) {
+                    if (!SL && h <= H) {
                         int mine = L[0][h];
 #pragma unroll
                         for (int w = 1; w < GW; ++w) if (set == w) mine = L[w][h];
@@ -717,8 +804,13 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 #pragma unroll
                     for (int w = 0; w < GW; ++w) {
                         int mm = Mh[0] - L[w][0];
+                        if (SL) {
+                            const int g = lane + 32 * w;
+                            if (g < G)
+                                for (int h = 1; h <= H; ++h) mm = min(mm, M_s[h] - L_s[g * H1 + h]);
+                        }
 #pragma unroll
-                        for (int h = 1; h <= HM; ++h) if (h <= H) mm = min(mm, Mh[h] - L[w][h]);
+                        for (int h = 1; h <= HR; ++h) if (h <= H) mm = min(mm, Mh[h] - L[w][h]);
                         if (cap[w] > 0 && (cap[w] > bc || (cap[w] == bc && mm > bm))) { bc = cap[w]; bm = mm; bg = lane + 32 * w; }
                     }
                     const int mc = __reduce_max_sync(kFull, bc);

@@ -233,3 +233,31 @@ def test_brh_random_shapes():
                              arrival=("const", float(rng.choice([1.0, 8.0, 30.0]))), first_seed=5000 * case)
         run_parity(cfg, 2, 40, threads=int(rng.choice([0, 32, 64, 128])), check_every=10,
                    launch_steps=int(rng.choice([1, 1, 4])))
+
+
+@pytest.mark.parametrize("H,G,kw", [
+    (80, 8, dict(beta=48.0, gamma=0.9, W=256, init_queue=256)),                       # the paper's deployed lookahead and fleet
+    (80, 16, dict(gate=0.0, delta_T=1)),                              # every request refreshed every step
+    (40, 64, dict(B=32, init_active=30, W=400, init_queue=390, term_mode=1, hazard=0.01, gate=0.3)),  # two workers per router lane
+    (17, 5, dict(B=16, init_active=9, W=64, init_queue=40, S_greedy=0)),                           # just beyond the register-resident horizons
+])
+def test_long_horizons(H, G, kw):
+    """Horizons beyond 16 offsets keep projected loads, envelope and margins in shared memory."""
+    run_parity(wlm.get_config("c2", H=H, G=G, **kw), 2, 60, check_every=10, fscore=(G == 8))
+
+
+def test_long_horizon_multi_step_and_random_shapes():
+    rng = np.random.default_rng(808)
+    for case in range(6):
+        G = int(rng.integers(1, 65)); B = 8 * int(rng.integers(1, 9)); W = 4 * int(rng.integers(1, 100))
+        H = int(rng.integers(17, 81))
+        cfg = wlm.get_config("c2", G=G, B=B, W=W, H=H, R_max=int(rng.integers(1, 6)),
+                             S_greedy=int(rng.choice([-1, 0, G, 1 << 20])), delta_T=int(rng.choice([-1, 1, 7])),
+                             gate=float(rng.choice([0.0, 0.5, 0.9])), beta=float(rng.choice([1.0, 24.0, 96.0])),
+                             gamma=float(rng.choice([0.5, 0.9, 1.0])),
+                             init_active=int(rng.integers(0, B + 1)), init_queue=int(rng.integers(0, W + 1)),
+                             term_mode=int(rng.choice([1, 2])), hazard=float(rng.choice([0.002, 0.05])),
+                             beta_ab=(2.0, float(rng.choice([20.0, 50.0, 200.0]))),
+                             arrival=("const", float(rng.choice([1.0, 8.0]))), first_seed=7000 * case)
+        run_parity(cfg, 2, 30, threads=int(rng.choice([0, 32, 128])), check_every=10,
+                   launch_steps=int(rng.choice([1, 3])))
