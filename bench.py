@@ -608,7 +608,10 @@ def extras(torch, device, args, peak, peak_kind, summary):
         ex["entry_points"] = {"error": repr(e)}
     # latency path: one instance, one graph-replayed step per decode step
     lat = [latency_path(torch, "c1", device, 2000), latency_path(torch, "c2", device, 2000),
-           latency_path(torch, "c4", device, 1000)]
+           latency_path(torch, "c4", device, 1000), latency_path(torch, "h80", device, 1500)]
+    # the paper's own figure for its Python dispatcher at the same H, G and R_max (Section 5.3
+    # "Dispatch overhead", another machine and language): context, not a target
+    lat[3]["paper_dispatcher_tick_p50_us"] = 1200.0
     ex["latency"] = lat
     summary["latency_device_p50_us"] = {f"{l['workload']}(G={l['G']},W={l['W']},H={l['H']})": round(l["device_p50_us"], 1)
                                         for l in lat}
@@ -626,7 +629,8 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
     out = r.outputs(1)
     probs = None
     seeds_t = tab_t = None
-    if cfg.H > 0:
+    need_probs = cfg.H > 0 and cfg.pred_mode == 0          # the perfect-lookahead predictor reads no classifier rows
+    if need_probs:
         seeds_t = torch.from_numpy(wl.seeds.astype(np.int64)).to(device)
         tab_t = torch.from_numpy(wl.beta_tab).to(device)
         probs = wlm.term_probs_torch(wl, 0, device, seeds_t=seeds_t, tab_t=tab_t).contiguous()
@@ -635,7 +639,7 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
     for k in range(steps):
-        if cfg.H > 0:
+        if need_probs:
             wlm.term_probs_torch(wl, k, device, seeds_t=seeds_t, tab_t=tab_t, out=probs)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -651,7 +655,7 @@ def latency_path(torch, cfg_name, device, steps, overrides=None):
     acc = np.zeros(8)
     n_ph = 200
     for k in range(steps, steps + n_ph):
-        if cfg.H > 0:
+        if need_probs:
             wlm.term_probs_torch(wl, k, device, seeds_t=seeds_t, tab_t=tab_t, out=probs)
         r.step(st, out, probs)
         torch.cuda.synchronize()

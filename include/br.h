@@ -28,7 +28,7 @@
 extern "C" {
 #endif
 
-#define BR_VERSION 101
+#define BR_VERSION 102
 
 /* status codes returned by every entry point */
 #define BR_OK        0
@@ -71,7 +71,9 @@ typedef struct {
     int32_t score_mode;     /* 0: Eq. 1 in integers (needs H == 0); 1: Eq. 2 in fp64; < 0 -> 0 if H == 0 else 1 */
     int32_t term_mode;      /* 0: requests never end; 1: every slot ends with the same probability p per
                                step, independently (term_cdf); 2: end when a 24-bit Philox uniform <
-                               term_probs[slot][0]                                              */
+                               term_probs[slot][0]; 3: every request carries its output length o_i
+                               (Section 2.2): admitted at step x it runs at steps x .. x + o_i - 1
+                               (act_end, waiting_queue.o, out_tab)                              */
     const uint32_t *term_cdf; /* device [B], term_mode 1: term_cdf[j] = floor(2^32 (1 - (1-p)^(j+1))), the
                                CDF of the number of slots skipped before the next ending one.  Per
                                worker and step the ending slots are walked by these gaps: draw t is
@@ -85,6 +87,13 @@ typedef struct {
     int32_t s_max;          /* largest prompt length the caller will ever enqueue (range proof) */
     int32_t threads;        /* threads per instance (multiple of 32, <= 256); <= 0 -> chosen from G*B, H and the batch size */
     int32_t inst_per_block; /* instances per thread block when an instance runs on one warp (1..8); <= 0 -> 4 */
+    int32_t pred_mode;      /* H > 0 only.  0: c_hat from the classifier output term_probs (Eqs. 3-5 and the
+                               refresh rules); 1: c_hat = min(r_i(k), H) from the known lifetimes, the
+                               perfect-lookahead reference of Section 5.1 "Our methods" (needs term_mode 3;
+                               term_probs, act_chat0 and act_kref are not used and may be NULL)        */
+    const int32_t *out_tab; /* device [2^out_tab_log2] inverse-CDF table of output lengths o_i >= 1 given to
+                               arrivals in term_mode 3: word j % 4 of the Philox block (k, j / 4, 3, 0) */
+    int32_t out_tab_log2;
 } br_params;
 
 /* running requests; instance i occupies row first_instance + i of every array */
@@ -97,6 +106,8 @@ typedef struct {
     uint32_t *act_id;     /* [N][G][B] request id per slot; may be NULL                         */
     float    *act_chat0;  /* [N][G][B] c_hat at the last refresh (H > 0 only, else may be NULL) */
     uint8_t  *act_kref;   /* [N][G][B] step of the last refresh modulo 256 (H > 0 only)         */
+    int32_t  *act_end;    /* [N][G][B] term_mode 3: the step at whose end the request finishes
+                                       (x_i + o_i - 1); else may be NULL                         */
     int32_t  *step;       /* [N]      decode step k                                             */
     uint64_t *seed;       /* [N]      Philox key of the instance                                */
     uint32_t *next_id;    /* [N]      id given to the next arrival                              */
@@ -107,6 +118,8 @@ typedef struct {
     int32_t  *s;          /* [N][W] prompt length s_i = w_i^(1)                                 */
     uint32_t *id;         /* [N][W] request id                                                  */
     int32_t  *n;          /* [N]    current length                                              */
+    int32_t  *o;          /* [N][W] term_mode 3: output length o_i of the waiting request (latent to
+                                    the router, carried along for the simulation); else may be NULL */
 } br_waiting_queue;
 
 typedef struct {

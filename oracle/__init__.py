@@ -39,6 +39,7 @@ class OrcParams(C.Structure):
         ("arr_cdf", C.c_void_p), ("arr_len", C.c_int32), ("arr_period", C.c_int32),
         ("len_tab", C.c_void_p), ("len_tab_log2", C.c_int32),
         ("burst_every", C.c_int32), ("burst_size", C.c_int32), ("router", C.c_int32),
+        ("pred_mode", C.c_int32), ("out_tab", C.c_void_p), ("out_tab_log2", C.c_int32),
     ]
 
 
@@ -54,6 +55,8 @@ def lib():
         L.orc_destroy.argtypes = [C.c_void_p]
         L.orc_set_state.argtypes = [C.c_void_p, C.c_int32, C.c_uint32] + [C.c_void_p] * 6 + [C.c_int32]
         L.orc_get_state.argtypes = [C.c_void_p] + [C.c_void_p] * 10
+        L.orc_set_lifetimes.argtypes = [C.c_void_p] * 3
+        L.orc_get_lifetimes.argtypes = [C.c_void_p] * 3
         L.orc_step.argtypes = [C.c_void_p] + [C.c_void_p] * 5
         L.orc_route_only.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_projection.argtypes = [C.c_void_p] + [C.c_void_p] * 3
@@ -178,7 +181,7 @@ class Instance:
     def __init__(self, *, G, H, B, W, R_max=4, S_greedy=None, alpha=1.0, beta=None, gamma=1.0,
                  delta_T=None, gate=0.5, c_floor=1.0, score_mode=None, term_mode=0,
                  term_cdf=None, arr_rows=None, len_tab=None, burst_every=0, burst_size=0,
-                 router=0, seed=0):
+                 router=0, seed=0, pred_mode=0, out_tab=None):
         self.G, self.H, self.B, self.W = G, H, B, W
         self._arr = np.ascontiguousarray(
             arr_rows if arr_rows is not None else np.full((1, 1), 0xFFFFFFFF), dtype=np.uint32)
@@ -189,6 +192,10 @@ class Instance:
         assert self._term.shape == (B,)
         log2 = int(self._len.size).bit_length() - 1
         assert 1 << log2 == self._len.size
+        self._out = np.ascontiguousarray(
+            out_tab if out_tab is not None else np.ones(2, dtype=np.int32), dtype=np.int32)
+        olog2 = int(self._out.size).bit_length() - 1
+        assert 1 << olog2 == self._out.size
         p = OrcParams(
             G=G, H=H, B=B, W=W, R_max=R_max, S_greedy=2 * G if S_greedy is None else S_greedy,
             alpha=alpha, beta=float(G) if beta is None else beta, gamma=gamma,
@@ -197,7 +204,8 @@ class Instance:
             term_mode=term_mode, term_cdf=self._term.ctypes.data,
             arr_cdf=self._arr.ctypes.data, arr_len=self._arr.shape[1],
             arr_period=self._arr.shape[0], len_tab=self._len.ctypes.data, len_tab_log2=log2,
-            burst_every=burst_every, burst_size=burst_size, router=router)
+            burst_every=burst_every, burst_size=burst_size, router=router,
+            pred_mode=pred_mode, out_tab=self._out.ctypes.data, out_tab_log2=olog2)
         self.params = p
         self._h = lib().orc_create(C.byref(p), C.c_uint64(int(seed)))
 
@@ -219,6 +227,18 @@ class Instance:
         qi = None if wq_id is None else np.ascontiguousarray(wq_id, dtype=np.uint32)
         lib().orc_set_state(self._h, int(k), int(next_id), _p(ab), _p(ai), _p(ch), _p(ta),
                             _p(qs), _p(qi), int(wq_n))
+
+    def set_lifetimes(self, act_end, wq_o):
+        """term_mode 3: the step at whose end each running request finishes, and the output
+        lengths of the waiting requests (call after set_state)."""
+        ae = np.ascontiguousarray(act_end, dtype=np.int32).reshape(self.G * self.B)
+        qo = np.ascontiguousarray(wq_o, dtype=np.int32).reshape(self.W)
+        lib().orc_set_lifetimes(self._h, _p(ae), _p(qo))
+
+    def get_lifetimes(self):
+        ae = np.zeros(self.G * self.B, dtype=np.int32); qo = np.zeros(self.W, dtype=np.int32)
+        lib().orc_get_lifetimes(self._h, _p(ae), _p(qo))
+        return ae.reshape(self.G, self.B), qo
 
     def get_state(self) -> Dict[str, np.ndarray]:
         A = self.G * self.B
@@ -284,7 +304,7 @@ def instance_from_workload(wl, inst: int, router: int = 0, **overrides) -> Insta
               gate=cfg.gate, c_floor=cfg.c_floor, score_mode=cfg.score_mode,
               term_mode=cfg.term_mode, term_cdf=wl.term_cdf, arr_rows=wl.arr_rows_for(inst),
               len_tab=wl.len_tab, burst_every=cfg.burst_every, burst_size=cfg.burst_size,
-              router=router, seed=int(wl.seeds[inst]))
+              router=router, seed=int(wl.seeds[inst]), pred_mode=cfg.pred_mode, out_tab=wl.out_tab)
     if cfg.score_mode == 0:
         kw["beta"] = float(cfg.G)
         kw["alpha"] = 1.0
@@ -295,4 +315,6 @@ def instance_from_workload(wl, inst: int, router: int = 0, **overrides) -> Insta
     chat, tau = explicit_pred_state(st["act_chat0"][inst], st["act_kref"][inst], k)
     o.set_state(k, int(st["next_id"][inst]), st["act_base"][inst], st["act_id"][inst], chat, tau,
                 st["wq_s"][inst], st["wq_id"][inst], int(st["wq_n"][inst]))
+    if "act_end" in st:
+        o.set_lifetimes(st["act_end"][inst], st["wq_o"][inst])
     return o

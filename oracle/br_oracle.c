@@ -49,7 +49,8 @@ typedef struct {
     int32_t delta_T;
     float   gate, c_floor;
     int32_t score_mode;          /* 0: Eq. 1 in integers; 1: Eq. 2 in fp64          */
-    int32_t term_mode;           /* 0 none; 1 constant hazard; 2 Bernoulli(probs[.][0]) */
+    int32_t term_mode;           /* 0 none; 1 constant hazard; 2 Bernoulli(probs[.][0]);
+                                    3 every request carries its output length o_i (Section 2.2) */
     const uint32_t *term_cdf;    /* [B] gap thresholds of the constant hazard (term_mode 1) */
     const uint32_t *arr_cdf;     /* [arr_period][arr_len] rows for this instance    */
     int32_t arr_len, arr_period;
@@ -57,6 +58,11 @@ typedef struct {
     int32_t len_tab_log2;
     int32_t burst_every, burst_size;
     int32_t router;              /* 0 BalanceRoute; 1 round-robin; 2 least-loaded   */
+    int32_t pred_mode;           /* 0: c_hat from classifier output (Eqs. 3-5, refresh rules);
+                                    1: c_hat = min(r_i(k), H) from the known lifetimes, the
+                                       perfect-lookahead reference of Section 5.1 (term_mode 3) */
+    const int32_t *out_tab;      /* inverse-CDF table of output lengths (term_mode 3) */
+    int32_t out_tab_log2;
 } orc_params;
 
 typedef struct {
@@ -71,8 +77,10 @@ typedef struct {
     int64_t  *cur;
     float    *chat;
     int32_t  *tau;
+    int32_t  *kend;              /* term_mode 3: the step at whose end the request finishes */
     /* waiting requests in arrival order */
     int32_t  *qs;
+    int32_t  *qo;                /* term_mode 3: output length o_i of the waiting request */
     uint32_t *qid;
     uint8_t  *qgone;
     int32_t  qn;
@@ -107,7 +115,7 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2 };
+enum { STREAM_ARR_COUNT = 0, STREAM_ARR_LEN = 1, STREAM_TERM = 2, STREAM_ARR_OUT = 3 };
 
 static uint32_t draw(const orc_inst *s, uint32_t entity, uint32_t stream)
 {
@@ -248,7 +256,9 @@ orc_inst *orc_create(const orc_params *p, uint64_t seed)
     s->cur = (int64_t *)calloc(A, sizeof(int64_t));
     s->chat = (float *)calloc(A, sizeof(float));
     s->tau = (int32_t *)calloc(A, sizeof(int32_t));
+    s->kend = (int32_t *)calloc(A, sizeof(int32_t));
     s->qs = (int32_t *)calloc(p->W, sizeof(int32_t));
+    s->qo = (int32_t *)calloc(p->W, sizeof(int32_t));
     s->qid = (uint32_t *)calloc(p->W, sizeof(uint32_t));
     s->qgone = (uint8_t *)calloc(p->W, 1);
     s->Lh = (int64_t *)calloc((size_t)p->G * H1, sizeof(int64_t));
@@ -263,8 +273,8 @@ orc_inst *orc_create(const orc_params *p, uint64_t seed)
 void orc_destroy(orc_inst *s)
 {
     if (!s) return;
-    free(s->occ); free(s->sid); free(s->cur); free(s->chat); free(s->tau);
-    free(s->qs); free(s->qid); free(s->qgone);
+    free(s->occ); free(s->sid); free(s->cur); free(s->chat); free(s->tau); free(s->kend);
+    free(s->qs); free(s->qo); free(s->qid); free(s->qgone);
     free(s->Lh); free(s->Mh); free(s->m); free(s->cap); free(s->d);
     free(s);
 }
@@ -308,6 +318,22 @@ void orc_get_state(const orc_inst *s, int32_t *k, uint32_t *next_id,
     }
 }
 
+/* lifetimes (term_mode 3): act_end[slot] = step at whose end the request finishes, wq_o[i] =
+ * output length of waiting request i */
+void orc_set_lifetimes(orc_inst *s, const int32_t *act_end, const int32_t *wq_o)
+{
+    int A = s->p.G * s->p.B;
+    for (int a = 0; a < A; ++a) s->kend[a] = act_end[a];
+    for (int i = 0; i < s->qn; ++i) s->qo[i] = wq_o[i];
+}
+
+void orc_get_lifetimes(const orc_inst *s, int32_t *act_end, int32_t *wq_o)
+{
+    int A = s->p.G * s->p.B;
+    for (int a = 0; a < A; ++a) act_end[a] = s->kend[a];
+    for (int i = 0; i < s->qn; ++i) wq_o[i] = s->qo[i];
+}
+
 /* ------------------------------------------------------------------ */
 /* one decode step                                                     */
 /* ------------------------------------------------------------------ */
@@ -325,6 +351,8 @@ static void arrive(orc_inst *s)
         uint32_t r = draw(s, (uint32_t)j, STREAM_ARR_LEN);
         int32_t len = p->len_tab[r >> (32 - p->len_tab_log2)];
         if (s->qn < p->W) {
+            if (p->term_mode == 3)      /* the request's output length comes with it (latent to the router) */
+                s->qo[s->qn] = p->out_tab[draw(s, (uint32_t)j, STREAM_ARR_OUT) >> (32 - p->out_tab_log2)];
             s->qs[s->qn] = len;
             s->qid[s->qn] = s->next_id + (uint32_t)j;
             s->qn++;
@@ -341,6 +369,16 @@ static void predict(orc_inst *s, const float *probs)
     const orc_params *p = &s->p;
     int A = p->G * p->B;
     if (p->H == 0) return;
+    if (p->pred_mode == 1) {
+        /* perfect lookahead (Section 5.1 "Our methods", BR-H oracle): c_hat = min(r_i(k), H), where
+         * r_i(k) counts the steps the request still runs, this one included */
+        for (int a = 0; a < A; ++a) {
+            if (!s->occ[a]) continue;
+            int64_t r = (int64_t)s->kend[a] - s->k + 1;
+            s->chat[a] = (float)(r < p->H ? r : p->H);
+        }
+        return;
+    }
     for (int a = 0; a < A; ++a) {
         if (!s->occ[a]) continue;
         int32_t t = s->tau[a] + 1;
@@ -433,6 +471,7 @@ static void commit(orc_inst *s, int i, int g, int32_t *assign)
     s->occ[a] = 1; s->sid[a] = s->qid[i]; s->cur[a] = s->qs[i];     /* w^(1) = s_i */
     s->chat[a] = (float)p->H;
     s->tau[a] = p->delta_T - 1;           /* READING: first prediction at the next step */
+    if (p->term_mode == 3) s->kend[a] = s->k + s->qo[i] - 1;   /* runs at steps k .. k + o_i - 1 */
     s->qgone[i] = 1;
     s->cap[g]--;
     /* READING: the admitted request adds a constant s_i at every offset */
@@ -580,7 +619,7 @@ void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
     /* stable removal of admitted requests */
     int w = 0;
     for (int i = 0; i < s->qn; ++i)
-        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; ++w; }
+        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; s->qo[w] = s->qo[i]; ++w; }
     s->qn = w;
 
     /* RECORD: loads from scratch */
@@ -609,6 +648,8 @@ void orc_step(orc_inst *s, const float *probs, int32_t *assign, int64_t *load,
             } else if (p->term_mode == 2) {
                 uint32_t u = draw(s, (uint32_t)a, STREAM_TERM) >> 8;       /* 24 bits */
                 fin = ((float)u * 5.9604644775390625e-8f) < probs[(size_t)a * p->H];
+            } else if (p->term_mode == 3) {
+                fin = s->kend[a] == s->k;                                  /* its o_i-th step */
             }
             if (fin) { s->occ[a] = 0; s->cur[a] = 0; }
             else s->cur[a] += 1;
@@ -655,7 +696,7 @@ void orc_route_only(orc_inst *s, int32_t *assign, int64_t *loads_out)
     for (int g = 0; g < p->G; ++g) loads_out[g] = s->Lh[g * H1];
     int w = 0;
     for (int i = 0; i < s->qn; ++i)
-        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; ++w; }
+        if (!s->qgone[i]) { s->qs[w] = s->qs[i]; s->qid[w] = s->qid[i]; s->qo[w] = s->qo[i]; ++w; }
     s->qn = w;
 }
 

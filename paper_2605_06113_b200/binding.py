@@ -30,17 +30,18 @@ class BrParams(C.Structure):
         ("len_tab", C.c_void_p), ("len_tab_log2", C.c_int32),
         ("burst_every", C.c_int32), ("burst_size", C.c_int32),
         ("s_max", C.c_int32), ("threads", C.c_int32), ("inst_per_block", C.c_int32),
+        ("pred_mode", C.c_int32), ("out_tab", C.c_void_p), ("out_tab_log2", C.c_int32),
     ]
 
 
 class BrWorkerState(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
-                ("load", "nact", "occ", "act_base", "act_id", "act_chat0", "act_kref",
+                ("load", "nact", "occ", "act_base", "act_id", "act_chat0", "act_kref", "act_end",
                  "step", "seed", "next_id")]
 
 
 class BrWaitingQueue(C.Structure):
-    _fields_ = [("s", C.c_void_p), ("id", C.c_void_p), ("n", C.c_void_p)]
+    _fields_ = [("s", C.c_void_p), ("id", C.c_void_p), ("n", C.c_void_p), ("o", C.c_void_p)]
 
 
 class BrInstanceBatch(C.Structure):
@@ -121,7 +122,8 @@ def _to_torch(a: np.ndarray, device):
 
 _STATE_DTYPES = dict(load=np.int64, nact=np.int32, occ=np.uint64, act_base=np.int32,
                      act_id=np.uint32, act_chat0=np.float32, act_kref=np.uint8, step=np.int32,
-                     seed=np.uint64, next_id=np.uint32, wq_s=np.int32, wq_id=np.uint32, wq_n=np.int32)
+                     seed=np.uint64, next_id=np.uint32, wq_s=np.int32, wq_id=np.uint32, wq_n=np.int32,
+                     act_end=np.int32, wq_o=np.int32)
 
 
 class Router:
@@ -137,6 +139,7 @@ class Router:
         self.len_tab = _to_torch(wl.len_tab, self.device)
         self.arr_cdf = _to_torch(wl.arr_cdf, self.device)
         self.term_cdf = _to_torch(wl.term_cdf, self.device)
+        self.out_tab = _to_torch(wl.out_tab, self.device) if wl.out_tab is not None else None
         p = BrParams(
             B=cfg.B, W=cfg.W, R_max=cfg.R_max, S_greedy=cfg.S_greedy, alpha=cfg.alpha,
             beta=cfg.beta, gamma=cfg.gamma, delta_T=cfg.delta_T, gate=cfg.gate, c_floor=cfg.c_floor,
@@ -145,7 +148,9 @@ class Router:
             arr_inst_stride=wl.arr_inst_stride, len_tab=self.len_tab.data_ptr(),
             len_tab_log2=int(wl.len_tab.size).bit_length() - 1, burst_every=cfg.burst_every,
             burst_size=cfg.burst_size, s_max=int(max(cfg.len_clip[1], cfg.ctx_clip[1])),
-            threads=threads)
+            threads=threads, pred_mode=cfg.pred_mode,
+            out_tab=self.out_tab.data_ptr() if self.out_tab is not None else None,
+            out_tab_log2=int(wl.out_tab.size).bit_length() - 1 if wl.out_tab is not None else 0)
         for k, v in overrides.items():
             setattr(p, k, v)
         self.params = p
@@ -189,9 +194,9 @@ class Router:
 
     def _structs(self, st, out, N, first, n_steps, stream):
         ws = BrWorkerState(**{k: _ptr(st.get(k)) for k in
-                              ("load", "nact", "occ", "act_base", "act_id", "act_chat0", "act_kref",
+                              ("load", "nact", "occ", "act_base", "act_id", "act_chat0", "act_kref", "act_end",
                                "step", "seed", "next_id")})
-        wq = BrWaitingQueue(s=_ptr(st["wq_s"]), id=_ptr(st["wq_id"]), n=_ptr(st["wq_n"]))
+        wq = BrWaitingQueue(s=_ptr(st["wq_s"]), id=_ptr(st["wq_id"]), n=_ptr(st["wq_n"]), o=_ptr(st.get("wq_o")))
         lo = BrLoadOut(load=_ptr(out["load"]), trace=_ptr(out["trace"]), status=_ptr(out.get("status")),
                        counters=_ptr(out.get("counters")), fscore=_ptr(out.get("fscore")),
                        phase_cycles=_ptr(out.get("phase_cycles")))

@@ -86,13 +86,16 @@ int check_step_args(const br_ctx *ctx, const br_instance_batch *b, const br_work
         return BR_EINVAL;
     if (!wq->s || !wq->id || !wq->n) return BR_EINVAL;
     if (!assign_out || !out->load || !out->trace) return BR_EINVAL;
-    if (ctx->H > 0 && (!ws->act_chat0 || !ws->act_kref || !term_probs)) return BR_EINVAL;
+    const bool classifier = ctx->H > 0 && ctx->p.pred_mode == 0;
+    if (classifier && (!ws->act_chat0 || !ws->act_kref || !term_probs)) return BR_EINVAL;
     if (ctx->p.term_mode == 2 && !term_probs) return BR_EINVAL;
+    if (ctx->p.term_mode == 3 && (!ws->act_end || !wq->o || misaligned(ws->act_end, 16) || misaligned(wq->o, 16)))
+        return BR_EINVAL;
     if (misaligned(ws->act_base, 16) || misaligned(wq->s, 16) || misaligned(wq->id, 16) ||
         misaligned(assign_out, 16) || misaligned(ws->load, 8) || misaligned(ws->occ, 8) ||
         misaligned(out->load, 8) || misaligned(out->trace, 8) || misaligned(ws->seed, 8) ||
         (term_probs && misaligned(term_probs, 16)) || (out->fscore && misaligned(out->fscore, 8)) ||
-        (ctx->H > 0 && (misaligned(ws->act_chat0, 16) || misaligned(ws->act_kref, 4))))
+        (classifier && (misaligned(ws->act_chat0, 16) || misaligned(ws->act_kref, 4))))
         return BR_EINVAL;
     return BR_OK;
 }
@@ -212,8 +215,11 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     if (p.c_floor < 0.0f) p.c_floor = 1.0f;
     if (p.score_mode < 0) p.score_mode = (H == 0) ? 0 : 1;
     if (p.score_mode > 1 || (p.score_mode == 0 && H != 0)) return BR_EINVAL;
-    if (p.term_mode < 0 || p.term_mode > 2 || (p.term_mode == 2 && H == 0)) return BR_EINVAL;
+    if (p.term_mode < 0 || p.term_mode > 3 || (p.term_mode == 2 && H == 0)) return BR_EINVAL;
     if (p.term_mode == 1 && !p.term_cdf) return BR_EINVAL;
+    if (p.pred_mode < 0) p.pred_mode = 0;
+    if (p.pred_mode > 1 || (p.pred_mode == 1 && (H == 0 || p.term_mode != 3))) return BR_EINVAL;
+    if (p.term_mode == 3 && p.arr_cdf && (!p.out_tab || p.out_tab_log2 < 0 || p.out_tab_log2 > 24)) return BR_EINVAL;
     if (p.arr_cdf) {
         if (p.arr_len < 1 || p.arr_period < 1 || p.arr_inst_stride < 0 || !p.len_tab) return BR_EINVAL;
         if (p.len_tab_log2 < 0 || p.len_tab_log2 > 24) return BR_EINVAL;
@@ -260,6 +266,7 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     a.magic_B = (uint32_t)(((1ull << 32) + (unsigned)p.B - 1) / (unsigned)p.B);
     a.delta_T = p.delta_T; a.gate = p.gate; a.c_floor = p.c_floor;
     a.term_mode = p.term_mode; a.term_cdf = p.term_cdf;
+    a.pred_mode = p.pred_mode; a.out_tab = p.out_tab; a.out_shift = 32 - p.out_tab_log2;
     a.arr_cdf = p.arr_cdf; a.arr_len = p.arr_len; a.arr_period = p.arr_period;
     a.arr_inst_stride = p.arr_inst_stride;
     a.len_tab = p.len_tab; a.len_shift = 32 - p.len_tab_log2;
@@ -295,11 +302,11 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
     } else {
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G; a.peak_ok = 0;
     }
-    ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words);
+    ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words, p.term_mode == 3);
     if (ctx->smem > 227 * 1024) { delete ctx; return BR_EINVAL; }      // one instance must fit a thread block's shared memory
     // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 512 waiting requests,
     // arrivals served by one Philox call, and negative queue keys scoring below every waiting request
-    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode != 2 &&
+    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode <= 1 &&
                     p.burst_every == 0 && (!p.arr_cdf || p.arr_len <= 64) &&
                     (long long)(G - 1) * p.s_max + 65536 < (1ll << (31 - wl));
     *out = ctx;
@@ -346,55 +353,87 @@ int br_graph_step(br_ctx *ctx)
     return BR_OK;
 }
 
-int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *hws,
-                 br_waiting_queue *hwq, const float *h_probs, int32_t *h_assign, br_load_out *hout,
-                 int64_t *h2d_bytes, int64_t *d2h_bytes)
+namespace {
+
+// One block of the staging area of the host-buffer entry points: a [N][row] array that goes up
+// before the kernel (in), comes down after it (out), or both.
+struct StageBlk { size_t bytes; void **dev; void *host; bool in, out; };
+constexpr int kStageBlks = 23;
+
+struct StagePlan {
+    StageBlk blk[kStageBlks];
+    br_worker_state dws; br_waiting_queue dwq; br_load_out dout;
+    float *d_probs; int32_t *d_assign;
+    size_t total;               // bytes, every block padded to 256
+};
+
+// Validates the host pointers of a host-buffer step and lists its blocks (device addresses are
+// assigned by the caller once it knows where the staging area is).
+int plan_host_step(const br_ctx *ctx, const br_instance_batch *batch, br_worker_state *hws, br_waiting_queue *hwq,
+                   const float *h_probs, int32_t *h_assign, br_load_out *hout, StagePlan *pl)
 {
     if (!ctx || !batch || !hws || !hwq || !hout) return BR_EINVAL;
     if (batch->n_instances < 0 || batch->first_instance != 0 || batch->n_steps > 1) return BR_EINVAL;
     if (!hws->load || !hws->nact || !hws->occ || !hws->act_base || !hws->step || !hws->seed ||
         !hws->next_id || !hwq->s || !hwq->id || !hwq->n || !h_assign || !hout->load || !hout->trace)
         return BR_EINVAL;
-    if (ctx->H > 0 && (!hws->act_chat0 || !hws->act_kref || !h_probs)) return BR_EINVAL;
+    const bool pred = ctx->H > 0 && ctx->p.pred_mode == 0;
+    const bool life = ctx->p.term_mode == 3;
+    if (pred && (!hws->act_chat0 || !hws->act_kref || !h_probs)) return BR_EINVAL;
     if (ctx->p.term_mode == 2 && !h_probs) return BR_EINVAL;
+    if (life && (!hws->act_end || !hwq->o)) return BR_EINVAL;
     const size_t N = (size_t)batch->n_instances;
-    if (N == 0) return BR_OK;
     const size_t G = ctx->G, H = ctx->H, B = ctx->p.B, W = ctx->p.W, A = G * B;
     const size_t OW = (B + 63) / 64;
-    cudaStream_t st = (cudaStream_t)batch->stream;
-
-    // staging layout: every block padded to 256 bytes
-    struct Blk { size_t bytes; void **dev; void *host; bool in, out; };
-    br_worker_state dws; memset(&dws, 0, sizeof(dws));
-    br_waiting_queue dwq; memset(&dwq, 0, sizeof(dwq));
-    br_load_out dout; memset(&dout, 0, sizeof(dout));
-    float *d_probs = nullptr; int32_t *d_assign = nullptr;
-    const bool pred = H > 0;
-    Blk blks[] = {
-        {N * G * 8, (void **)&dws.load, hws->load, true, true},
-        {N * G * 4, (void **)&dws.nact, hws->nact, true, true},
-        {N * G * OW * 8, (void **)&dws.occ, hws->occ, true, true},
-        {N * A * 4, (void **)&dws.act_base, hws->act_base, true, true},
-        {hws->act_id ? N * A * 4 : 0, (void **)&dws.act_id, hws->act_id, true, true},
-        {pred ? N * A * 4 : 0, (void **)&dws.act_chat0, hws->act_chat0, true, true},
-        {pred ? N * A : 0, (void **)&dws.act_kref, hws->act_kref, true, true},
-        {N * 4, (void **)&dws.step, hws->step, true, true},
-        {N * 8, (void **)&dws.seed, hws->seed, true, false},
-        {N * 4, (void **)&dws.next_id, hws->next_id, true, true},
-        {N * W * 4, (void **)&dwq.s, hwq->s, true, true},
-        {N * W * 4, (void **)&dwq.id, hwq->id, true, true},
-        {N * 4, (void **)&dwq.n, hwq->n, true, true},
-        {h_probs ? N * A * H * 4 : 0, (void **)&d_probs, (void *)h_probs, true, false},
-        {N * W * 4, (void **)&d_assign, h_assign, false, true},
-        {N * G * 8, (void **)&dout.load, hout->load, false, true},
-        {N * 3 * 8, (void **)&dout.trace, hout->trace, false, true},
-        {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
-        {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
-        {hout->fscore ? N * W * G * 8 : 0, (void **)&dout.fscore, hout->fscore, false, true},
-        {hout->phase_cycles ? N * 32 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
+    memset(&pl->dws, 0, sizeof(pl->dws)); memset(&pl->dwq, 0, sizeof(pl->dwq)); memset(&pl->dout, 0, sizeof(pl->dout));
+    pl->d_probs = nullptr; pl->d_assign = nullptr;
+    const StageBlk blks[kStageBlks] = {
+        {N * G * 8, (void **)&pl->dws.load, hws->load, true, true},
+        {N * G * 4, (void **)&pl->dws.nact, hws->nact, true, true},
+        {N * G * OW * 8, (void **)&pl->dws.occ, hws->occ, true, true},
+        {N * A * 4, (void **)&pl->dws.act_base, hws->act_base, true, true},
+        {hws->act_id ? N * A * 4 : 0, (void **)&pl->dws.act_id, hws->act_id, true, true},
+        {pred ? N * A * 4 : 0, (void **)&pl->dws.act_chat0, hws->act_chat0, true, true},
+        {pred ? N * A : 0, (void **)&pl->dws.act_kref, hws->act_kref, true, true},
+        {life ? N * A * 4 : 0, (void **)&pl->dws.act_end, hws->act_end, true, true},
+        {N * 4, (void **)&pl->dws.step, hws->step, true, true},
+        {N * 8, (void **)&pl->dws.seed, hws->seed, true, false},
+        {N * 4, (void **)&pl->dws.next_id, hws->next_id, true, true},
+        {N * W * 4, (void **)&pl->dwq.s, hwq->s, true, true},
+        {N * W * 4, (void **)&pl->dwq.id, hwq->id, true, true},
+        {life ? N * W * 4 : 0, (void **)&pl->dwq.o, hwq->o, true, true},
+        {N * 4, (void **)&pl->dwq.n, hwq->n, true, true},
+        {h_probs ? N * A * H * 4 : 0, (void **)&pl->d_probs, (void *)h_probs, true, false},
+        {N * W * 4, (void **)&pl->d_assign, h_assign, false, true},
+        {N * G * 8, (void **)&pl->dout.load, hout->load, false, true},
+        {N * 3 * 8, (void **)&pl->dout.trace, hout->trace, false, true},
+        {hout->status ? N * 4 : 0, (void **)&pl->dout.status, hout->status, false, true},
+        {hout->counters ? N * 16 : 0, (void **)&pl->dout.counters, hout->counters, false, true},
+        {hout->fscore ? N * W * G * 8 : 0, (void **)&pl->dout.fscore, hout->fscore, false, true},
+        {hout->phase_cycles ? N * 32 : 0, (void **)&pl->dout.phase_cycles, hout->phase_cycles, false, true},
     };
-    size_t total = 0;
-    for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;
+    pl->total = 0;
+    for (int i = 0; i < kStageBlks; ++i) { pl->blk[i] = blks[i]; pl->total += (blks[i].bytes + 255) & ~(size_t)255; }
+    return BR_OK;
+}
+
+}  // namespace
+
+int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *hws,
+                 br_waiting_queue *hwq, const float *h_probs, int32_t *h_assign, br_load_out *hout,
+                 int64_t *h2d_bytes, int64_t *d2h_bytes)
+{
+    StagePlan pl;
+    int rc = plan_host_step(ctx, batch, hws, hwq, h_probs, h_assign, hout, &pl);
+    if (rc != BR_OK) return rc;
+    const size_t N = (size_t)batch->n_instances;
+    if (N == 0) return BR_OK;
+    cudaStream_t st = (cudaStream_t)batch->stream;
+    typedef StageBlk Blk;
+    Blk (&blks)[kStageBlks] = pl.blk;
+    br_worker_state &dws = pl.dws; br_waiting_queue &dwq = pl.dwq; br_load_out &dout = pl.dout;
+    float *&d_probs = pl.d_probs; int32_t *&d_assign = pl.d_assign;
+    const size_t total = pl.total;
     if (total > ctx->stage_bytes) {
         if (ctx->stage) { cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
         cudaError_t e = cudaMalloc(&ctx->stage, total);
@@ -411,7 +450,7 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         if (b.out) down += (int64_t)b.bytes;
     }
     br_instance_batch db = *batch; db.n_steps = 1;
-    int rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
+    rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
     if (rc != BR_OK) return rc;
     // Large batches go through in chunks of instances on three streams: the upload of chunk c + 1,
     // the kernel of chunk c and the download of chunk c - 1 overlap (the two copy directions use
@@ -511,54 +550,22 @@ int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_s
                         br_waiting_queue *hwq, const float *h_probs, int32_t *h_assign,
                         br_load_out *hout, int64_t *h2d_bytes, int64_t *d2h_bytes)
 {
-    if (!ctx || !batch || !hws || !hwq || !hout) return BR_EINVAL;
-    if (batch->n_instances < 0 || batch->first_instance != 0 || batch->n_steps > 1) return BR_EINVAL;
-    if (!hws->load || !hws->nact || !hws->occ || !hws->act_base || !hws->step || !hws->seed ||
-        !hws->next_id || !hwq->s || !hwq->id || !hwq->n || !h_assign || !hout->load || !hout->trace)
-        return BR_EINVAL;
-    if (ctx->H > 0 && (!hws->act_chat0 || !hws->act_kref || !h_probs)) return BR_EINVAL;
-    if (ctx->p.term_mode == 2 && !h_probs) return BR_EINVAL;
-    if (hout->fscore) return BR_EINVAL;                 // the score matrix is not offered on this path
+    if (hout && hout->fscore) return BR_EINVAL;         // the score matrix is not offered on this path
+    StagePlan pl;
+    int rc = plan_host_step(ctx, batch, hws, hwq, h_probs, h_assign, hout, &pl);
+    if (rc != BR_OK) return rc;
     const size_t N = (size_t)batch->n_instances;
     if (N == 0) return BR_OK;
-    const size_t G = ctx->G, H = ctx->H, B = ctx->p.B, W = ctx->p.W, A = G * B;
-    const size_t OW = (B + 63) / 64;
     cudaStream_t st = (cudaStream_t)batch->stream;
-
-    struct Blk { size_t bytes; void **dev; void *host; bool in, out; };
-    br_worker_state dws; memset(&dws, 0, sizeof(dws));
-    br_waiting_queue dwq; memset(&dwq, 0, sizeof(dwq));
-    br_load_out dout; memset(&dout, 0, sizeof(dout));
-    float *d_probs = nullptr; int32_t *d_assign = nullptr;
-    const bool pred = H > 0;
-    Blk blks[] = {
-        {N * G * 8, (void **)&dws.load, hws->load, true, true},
-        {N * G * 4, (void **)&dws.nact, hws->nact, true, true},
-        {N * G * OW * 8, (void **)&dws.occ, hws->occ, true, true},
-        {N * A * 4, (void **)&dws.act_base, hws->act_base, true, true},
-        {hws->act_id ? N * A * 4 : 0, (void **)&dws.act_id, hws->act_id, true, true},
-        {pred ? N * A * 4 : 0, (void **)&dws.act_chat0, hws->act_chat0, true, true},
-        {pred ? N * A : 0, (void **)&dws.act_kref, hws->act_kref, true, true},
-        {N * 4, (void **)&dws.step, hws->step, true, true},
-        {N * 8, (void **)&dws.seed, hws->seed, true, false},
-        {N * 4, (void **)&dws.next_id, hws->next_id, true, true},
-        {N * W * 4, (void **)&dwq.s, hwq->s, true, true},
-        {N * W * 4, (void **)&dwq.id, hwq->id, true, true},
-        {N * 4, (void **)&dwq.n, hwq->n, true, true},
-        {h_probs ? N * A * H * 4 : 0, (void **)&d_probs, (void *)h_probs, true, false},
-        {N * W * 4, (void **)&d_assign, h_assign, false, true},
-        {N * G * 8, (void **)&dout.load, hout->load, false, true},
-        {N * 3 * 8, (void **)&dout.trace, hout->trace, false, true},
-        {hout->status ? N * 4 : 0, (void **)&dout.status, hout->status, false, true},
-        {hout->counters ? N * 16 : 0, (void **)&dout.counters, hout->counters, false, true},
-        {hout->phase_cycles ? N * 32 : 0, (void **)&dout.phase_cycles, hout->phase_cycles, false, true},
-    };
-    size_t total = 0;
-    for (const Blk &b : blks) total += (b.bytes + 255) & ~(size_t)255;
+    typedef StageBlk Blk;
+    Blk (&blks)[kStageBlks] = pl.blk;
+    br_worker_state &dws = pl.dws; br_waiting_queue &dwq = pl.dwq; br_load_out &dout = pl.dout;
+    float *&d_probs = pl.d_probs; int32_t *&d_assign = pl.d_assign;
+    const size_t total = pl.total;
     if (total > (size_t)BR_STATIC_STAGE_BYTES) return BR_ELIMIT;      // nothing was touched
 
     void *stage = nullptr;
-    int rc = static_stage_address(&stage);
+    rc = static_stage_address(&stage);
     if (rc != BR_OK) return rc;
 
     size_t off = 0, out_begin = 0, out_end = 0;

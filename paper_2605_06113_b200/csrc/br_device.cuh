@@ -11,7 +11,7 @@ constexpr int32_t kEmpty = INT32_MIN;
 constexpr long long kNoKey = (long long)0x8000000000000000ull;
 constexpr int kNoIdx = 0x7FFFFFFF;
 
-enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2 };
+enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2, kStreamArrOut = 3 };
 
 // First statements of a step kernel: let the next kernel of the stream start becoming resident,
 // then wait until every earlier kernel of the stream has completed and flushed its writes

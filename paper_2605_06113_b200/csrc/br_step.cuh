@@ -29,6 +29,9 @@ struct StepArgs {
     int32_t delta_T;
     float gate, c_floor;
     int32_t term_mode;
+    int32_t pred_mode;          // 1: c_hat = min(remaining steps, H) from act_end (term_mode 3)
+    const int32_t *out_tab;     // output lengths of arrivals (term_mode 3)
+    int32_t out_shift;
     const uint32_t *term_cdf;   // [B] gap thresholds of the constant hazard
     const uint32_t *arr_cdf;
     int32_t arr_len, arr_period, arr_inst_stride;
@@ -49,7 +52,7 @@ struct StepArgs {
 };
 
 // shared-memory footprint of one instance (bytes), mirrored by the host
-__host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words)
+__host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words, bool lifetimes = false)
 {
     size_t n = 0;
     n += 4 * (size_t)W * 2;                      // q_key, q_id
@@ -60,6 +63,8 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     n += 8 * (size_t)(H + 1) + 4 * (size_t)((H + 2) / 2 * 2);   // md_s (fp64 margins of the selected worker), M_s (envelope)
     n += 2 * 96 + 2 * 32 + 64;                   // end_list, pre_list, scalars
     if (H > 0) n += 2 * (size_t)G * B;           // refresh_list
+    n = (n + 15) & ~(size_t)15;
+    if (lifetimes) n += 4 * (size_t)W;           // q_o (output lengths of the waiting requests)
     return (n + 15) & ~(size_t)15;
 }
 
@@ -212,6 +217,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned short *pre_list = end_list + kEndList;                                 // [32]
     int *scal = reinterpret_cast<int *>(pre_list + 32);
     unsigned short *refresh_list = reinterpret_cast<unsigned short *>(scal + 16);   // [A] (H > 0 only)
+    // output lengths of the waiting requests (term_mode 3 only), behind everything else
+    int *q_o = reinterpret_cast<int *>(smem_raw + ((step_smem_bytes(G, H, B, W, OW) + 15) & ~(size_t)15));
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
     //       [6] requests that ended this step and were not prefetched, [7] prefetched ones,
@@ -225,6 +232,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     uint32_t *g_aid = a.ws.act_id ? a.ws.act_id + (size_t)inst * A : nullptr;
     float *g_chat0 = a.ws.act_chat0 ? a.ws.act_chat0 + (size_t)inst * A : nullptr;
     uint8_t *g_kref = a.ws.act_kref ? a.ws.act_kref + (size_t)inst * A : nullptr;
+    const bool life = !LEAN && a.term_mode == 3;          // requests carry their output lengths
+    int32_t *g_end = life ? a.ws.act_end + (size_t)inst * A : nullptr;
+    int32_t *g_qo = life ? a.wq.o + (size_t)inst * W : nullptr;
     int32_t *g_qs = a.wq.s + (size_t)inst * W;
     uint32_t *g_qid = a.wq.id + (size_t)inst * W;
 
@@ -249,6 +259,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         kk.w = (v.w << WL) | (int)(posmask - (unsigned)(i + 3));
         *reinterpret_cast<int4 *>(q_key + i) = kk;
         *reinterpret_cast<uint4 *>(q_id + i) = u;
+        if (life) *reinterpret_cast<int4 *>(q_o + i) = *reinterpret_cast<const int4 *>(g_qo + i);
     };
     {
         const int i0 = tid * 4, i1 = (NT + tid) * 4;
@@ -372,6 +383,10 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 const int s = a.len_tab[word_of(r, j & 3) >> a.len_shift];
                 q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
                 q_id[pos] = id0 + (unsigned)j;
+                if (life) {
+                    const uint4 ro = philox4x32_10((uint32_t)k, (uint32_t)j >> 2, kStreamArrOut, 0u, key0, key1);
+                    q_o[pos] = a.out_tab[word_of(ro, j & 3) >> a.out_shift];
+                }
             }
         }
         int n_drop = n_w + n_arr - W;
@@ -385,7 +400,27 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // the buckets into L_g(k+h) = sum_{j >= h} T_j + h * sum_{j >= h} C_j by suffix sums.
         // Pass A streams the per-request state and settles the requests that only age; the ones due
         // for a refresh are listed, and pass B reads their classifier rows with independent loads.
-        if (HM > 0 && H > 0) {
+        if (HM > 0 && H > 0 && !LEAN && a.pred_mode == 1) {
+            // perfect lookahead: c_hat = min(r_i(k), H) with r_i(k) = act_end - k + 1 steps still to run
+            const int A4 = A >> 2;
+#pragma unroll 2
+            for (int q4 = tid; q4 < A4; q4 += NT) {
+                const int4 bq = *reinterpret_cast<const int4 *>(g_base + 4 * q4);
+                const int4 eq = *reinterpret_cast<const int4 *>(g_end + 4 * q4);
+                const int bs4[4] = {bq.x, bq.y, bq.z, bq.w};
+                const int en4[4] = {eq.x, eq.y, eq.z, eq.w};
+                const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (bs4[j] != kEmpty) {
+                        int nh = en4[j] - k + 1;
+                        nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                        atomicAdd(&Lh_s[g * H1 + nh], (unsigned)(bs4[j] + k));
+                        atomicAdd(&Ch_s[g * H1 + nh], 1u);
+                    }
+                }
+            }
+        } else if (HM > 0 && H > 0) {
             const int A4 = A >> 2;
 #pragma unroll 1
             for (int q_base = 0; q_base < A4; q_base += NT * kUnroll) {
@@ -721,10 +756,11 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         occ[g * OW + (slot >> 6)] |= 1ull << (slot & 63);
                         const int sa = g * B + slot;
                         g_base[sa] = s - k;
-                        if (H > 0) {
+                        if (H > 0 && g_chat0) {
                             g_chat0[sa] = (float)(H + a.delta_T - 1);
                             g_kref[sa] = (uint8_t)((k + 1 - a.delta_T) & 255);
                         }
+                        if (life) g_end[sa] = k + q_o[pos] - 1;          // runs at steps k .. k + o_i - 1
                         if (g_aid) g_aid[sa] = q_id[pos];
                         q_key[pos] = (int)(0x80000000u | (unsigned)sa);
                     } else {
@@ -969,6 +1005,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 const bool inq = i < n_before;
                 const int qk = inq ? q_key[i] : 0;
                 const unsigned id = inq ? q_id[i] : 0u;
+                const int qo = (life && inq) ? q_o[i] : 0;
                 const bool gone = inq && qk < 0;
                 const bool keep = inq && qk > 0;
                 const unsigned bal = __ballot_sync(kFull, keep);
@@ -994,6 +1031,10 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int s = qk >> WL;
                     if (dst != i) { q_key[dst] = (s << WL) | (int)(posmask - (unsigned)dst); q_id[dst] = id; }
                     if (dst != i || i >= n_w_old) { g_qs[dst] = s; g_qid[dst] = id; }
+                    if (life) {
+                        if (dst != i) q_o[dst] = qo;
+                        if (dst != i || i >= n_w_old) g_qo[dst] = qo;
+                    }
                 }
                 __syncwarp();
                 run += __popc(bal);
@@ -1032,6 +1073,24 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                                 if (__fmul_rn((float)(rr[j] >> 8), sc24) < q) fb |= 1u << jj;
                             }
                         }
+                    }
+                    reinterpret_cast<unsigned char *>(fin_w + (size_t)g * OW)[slot0 >> 3] = (unsigned char)fb;
+                }
+                inst_sync();
+            } else if (term_mode == 3) {
+                // a request ends with its o_i-th step: act_end == k
+#pragma unroll 1
+                for (int q8 = tid; q8 < A8; q8 += NT) {
+                    const int a0 = q8 << 3;
+                    const int g = a0 / B, slot0 = a0 - g * B;
+                    const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
+                    unsigned fb = 0;
+                    if (ob) {
+                        const int4 e0 = *reinterpret_cast<const int4 *>(g_end + a0);
+                        const int4 e1 = *reinterpret_cast<const int4 *>(g_end + a0 + 4);
+                        const int en[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) if (((ob >> j) & 1u) && en[j] == k) fb |= 1u << j;
                     }
                     reinterpret_cast<unsigned char *>(fin_w + (size_t)g * OW)[slot0 >> 3] = (unsigned char)fb;
                 }

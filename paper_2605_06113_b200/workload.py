@@ -33,6 +33,8 @@ STREAM_INIT_QUEUE = 2
 STREAM_INIT_TAU = 3
 STREAM_PROBS = 4
 STREAM_RATE = 5
+STREAM_INIT_END = 6
+STREAM_INIT_QO = 7
 
 _M1 = 0xBF58476D1CE4E5B9
 _M2 = 0x94D049BB133111EB
@@ -146,7 +148,8 @@ class Config:
     len_sigma: float
     arrival: Tuple                # ("const", lam) | ("sin", base, amp, period) | ("uniform", lo, hi)
     hazard: float                 # per-step termination probability (term_mode 1)
-    term_mode: int = 1            # 0 none, 1 constant hazard, 2 Bernoulli(term_probs[slot][0])
+    term_mode: int = 1            # 0 none, 1 constant hazard, 2 Bernoulli(term_probs[slot][0]),
+                                  # 3 every request carries its output length (out_mu, out_sigma)
     B: int = 64
     R_max: int = 4
     S_greedy: int = -1            # -1 -> 2 G
@@ -162,6 +165,10 @@ class Config:
     burst_size: int = 0
     len_clip: Tuple[int, int] = (1, 131072)
     ctx_clip: Tuple[int, int] = (16, 32768)
+    pred_mode: int = 0            # 0 classifier rows (term_probs), 1 perfect lookahead min(r_i, H) (needs term_mode 3)
+    out_mu: float = 6.5           # output lengths (decode steps) of term_mode 3: lognormal, clipped
+    out_sigma: float = 1.0
+    out_clip: Tuple[int, int] = (1, 32768)
 
     def resolved(self) -> "Config":
         c = self
@@ -192,6 +199,14 @@ CONFIGS: Dict[str, Config] = {
     "c3": Config("c3", N=4096, G=32, W=256, H=0, steps=500, first_seed=100, init_active=32,
                  init_queue=256, len_mu=7.5, len_sigma=1.2, arrival=("uniform", 4.0, 16.0),
                  hazard=1.0 / 500.0, ctx_clip=(16, 131072)),
+    # The paper's deployed setting (Section 5.1 "Our methods", Section 5.3 "Dispatch overhead"):
+    # BR-H with H = 80 on G = 8 workers, R_max = 4, perfect-lookahead predictor from simulated
+    # lifetimes; prompt and output lengths shaped like its traces (mean prompt ~4,000, mean output
+    # ~1,100 tokens), near saturation
+    "h80": Config("h80", N=1, G=8, W=512, H=80, steps=2000, first_seed=9000, init_active=64,
+                  init_queue=64, len_mu=8.0, len_sigma=0.8, arrival=("const", 0.7),
+                  hazard=0.0, term_mode=3, pred_mode=1, beta=48.0, gamma=0.9,
+                  out_mu=6.5, out_sigma=1.0, ctx_clip=(16, 131072)),
     # BR-H batched, H=8, bursts of 200 every 250 steps, geometric mean 600
     "c4": Config("c4", N=1024, G=64, W=1024, H=8, steps=1000, first_seed=5000,
                  init_active=64, init_queue=1024, len_mu=8.0, len_sigma=1.5,
@@ -218,6 +233,7 @@ class Workload:
     arr_period: int
     arr_inst_stride: int          # row(inst, k) = inst * stride + k % period
     term_cdf: np.ndarray          # uint32 [B] gap thresholds of the constant hazard
+    out_tab: Optional[np.ndarray] = None   # int32 [2^16] output lengths (term_mode 3)
     state: Dict[str, np.ndarray] = field(default_factory=dict)
 
     def arr_rows_for(self, inst: int) -> np.ndarray:
@@ -291,6 +307,20 @@ def make_workload(cfg: Config, n_instances: Optional[int] = None,
     act_chat0 = np.full((N, G, B), float(H), dtype=np.float32)
     act_kref = ((-tau0) & 255).astype(np.uint8)
 
+    out_tab = None
+    extra = {}
+    if cfg.term_mode == 3:
+        # every request carries its output length; a running request has a uniformly drawn part
+        # of its own still ahead, a waiting one all of it
+        out_tab = lognormal_table(cfg.out_mu, cfg.out_sigma, *cfg.out_clip)
+        z = mix_np(seeds[:, None], STREAM_INIT_END, slot)
+        o_run = out_tab[_top16(z)].astype(np.int64)
+        frac = ((z >> np.uint64(16)) & np.uint64(0xFFFF)).astype(np.int64)
+        act_end = ((o_run * frac) >> 16).reshape(N, G, B)            # last step of the request, in [0, o)
+        extra["act_end"] = np.where(occupied, act_end, 0).astype(np.int32)
+        q_o = out_tab[_top16(mix_np(seeds[:, None], STREAM_INIT_QO, qpos))].astype(np.int32)
+        extra["wq_o"] = np.where(q_valid, q_o, 0).astype(np.int32)
+
     state = dict(
         act_base=act_base, occ=occ, nact=nact, load=load, act_id=act_id,
         act_chat0=act_chat0, act_kref=act_kref,
@@ -299,9 +329,10 @@ def make_workload(cfg: Config, n_instances: Optional[int] = None,
         seed=seeds.copy(),
         next_id=np.full((N,), A + cfg.init_queue, dtype=np.uint32),
     )
+    state.update(extra)
     return Workload(cfg=cfg, seeds=seeds, len_tab=len_tab, beta_tab=btab, arr_cdf=arr,
                     arr_period=period, arr_inst_stride=stride,
-                    term_cdf=termination_gap_thresholds(cfg.hazard, B), state=state)
+                    term_cdf=termination_gap_thresholds(cfg.hazard, B), out_tab=out_tab, state=state)
 
 
 # --------------------------------------------------------------------------

@@ -27,7 +27,11 @@ def compare_state(cfg, st_np, o, i, k):
     assert int(st_np["wq_n"][i]) == n
     assert np.array_equal(st_np["wq_s"][i][:n], s["wq_s"][:n])
     assert np.array_equal(st_np["wq_id"][i][:n], s["wq_id"][:n])
-    if cfg.H > 0:
+    if cfg.term_mode == 3:
+        ae, qo = o.get_lifetimes() if hasattr(o, "get_lifetimes") else (s["act_end"], s["wq_o"])
+        assert np.array_equal(st_np["act_end"][i][occ], ae[occ]), f"act_end inst {i} step {k}"
+        assert np.array_equal(st_np["wq_o"][i][:n], qo[:n])
+    if cfg.H > 0 and cfg.pred_mode == 0:
         chat, tau = oracle.explicit_pred_state(st_np["act_chat0"][i], st_np["act_kref"][i], k)
         assert np.array_equal(chat[occ], s["chat"][occ]), f"c_hat inst {i} step {k}"
         assert np.array_equal(tau[occ], s["tau"][occ])

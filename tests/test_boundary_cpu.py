@@ -27,7 +27,7 @@ def test_library_exports_every_declared_entry_point():
     for n in names:
         assert hasattr(L, n), n
     assert sorted(binding.EXPORTS) == names
-    assert L.br_version() == 101
+    assert L.br_version() == 102
     assert L.br_strerror(BR_OK) == b"ok"
     assert b"invalid" in L.br_strerror(BR_EINVAL)
 
@@ -58,7 +58,7 @@ def test_create_validates_sizes_and_ranges():
     for G, H, kw in [(0, 0, {}), (65, 0, {}), (32, 81, {}), (32, -1, {}), (32, 0, dict(B=12)),
                      (32, 0, dict(B=264)), (32, 0, dict(W=6)), (32, 0, dict(W=8192)),
                      (32, 0, dict(R_max=6)), (32, 4, dict(score_mode=0)), (32, 0, dict(term_mode=2)),
-                     (32, 0, dict(term_mode=3)), (32, 0, dict(term_cdf=None)), (32, 4, dict(gamma=0.0)), (32, 4, dict(gamma=1.5)),
+                     (32, 0, dict(term_mode=4)), (32, 4, dict(pred_mode=1)), (32, 0, dict(term_mode=3, pred_mode=1)), (32, 0, dict(term_cdf=None)), (32, 4, dict(gamma=0.0)), (32, 4, dict(gamma=1.5)),
                      (32, 4, dict(alpha=-1.0)), (32, 0, dict(threads=48)), (32, 0, dict(threads=512)),
                      (32, 4, dict(delta_T=200))]:
         rc, h = _create(G, H, _params(**kw))
