@@ -44,7 +44,9 @@ extern "C" {
 #define BR_MAX_H      80     /* the lookahead the paper deploys (Section 5.1 "Our methods")   */
 #define BR_MAX_B     256     /* B must be a multiple of 8                     */
 #define BR_MAX_W    4096     /* W must be a multiple of 4                     */
-#define BR_MAX_RMAX    5     /* Stage 2 enumerates 2^R_max - 1 <= 31 subsets   */
+#define BR_MAX_RMAX   16     /* Stage-2 window; beyond 5 entries the subsets are searched by
+                                meeting in the middle, which needs G >= 2 (Eq. 1) or Eq. 2
+                                parameters without a flat segment and H <= 16       */
 
 #define BR_EMPTY_SLOT INT32_MIN  /* act_base value of a free slot              */
 
@@ -62,7 +64,7 @@ typedef struct br_ctx br_ctx;
 typedef struct {
     int32_t B;              /* slots per worker (max concurrency B, Section 2.2)             */
     int32_t W;              /* capacity of the waiting queue                                  */
-    int32_t R_max;          /* Stage-2 window (Algorithm 1); <= 0 -> 4                       */
+    int32_t R_max;          /* Stage-2 window (Algorithm 1); <= 0 -> 4; at most BR_MAX_RMAX  */
     int32_t S_greedy;       /* Stage-1 / Stage-2 threshold on total free slots; < 0 -> 2 G   */
     double  alpha, beta, gamma; /* Eq. 2 parameters; ignored when score_mode == 0            */
     int32_t delta_T;        /* c_hat refresh period; <= 0 -> max(1, H / 2)                   */
@@ -239,15 +241,21 @@ int br_fscore(br_ctx *ctx, const br_instance_batch *batch, const int32_t *s, int
               const int64_t *Lh, const int32_t *cap, double *F, int32_t *best_g);
 
 /*
- * The Stage-2 subproblem alone, solved exactly for windows larger than the R_max <= 5 of br_step
- * (Algorithms 1 and 2, Stage 2; Appendix "Bit-set subset selection": the score depends on Q only
- * through Delta(Q)).  For each of batch.n_instances problems: win [N][R] holds the prompt lengths
- * of the window (1 <= R <= 20; bit j of a mask selects entry j), margins [N][H+1] the worker's
- * m_{g,h} (H = 0: m_g), lim [N] the largest subset size (the worker's free slots).  Writes
- * best_mask [N] = the non-empty subset with |Q| <= lim and the highest F_g(Q) (Eq. 1 / Eq. 2 as
- * in br_step), lowest mask on ties, 0 if lim < 1; best_F [N] (may be NULL) its score.  All 2^R - 1
- * subsets are enumerated, one thread block per problem.  Device pointers; asynchronous on
- * batch.stream; BR_EINVAL for null pointers or R outside [1, 20].
+ * The Stage-2 subproblem alone, solved exactly on windows of up to 32 requests (Algorithms 1 and 2,
+ * Stage 2; Appendix "Bit-set subset selection": the score depends on Q only through Delta(Q)).
+ * For each of batch.n_instances problems: win [N][R] holds the prompt lengths of the window
+ * (1 <= R <= 32; bit j of a mask selects entry j), margins [N][H+1] the worker's m_{g,h} (H = 0:
+ * m_g), lim [N] the largest subset size (the worker's free slots).  Writes best_mask [N] = the
+ * non-empty subset with |Q| <= lim and the highest F_g(Q) (Eq. 1 / Eq. 2 as in br_step), lowest mask
+ * on ties, 0 if lim < 1; best_F [N] (may be NULL) its score.  Up to 12 requests all 2^R - 1 subsets
+ * are enumerated; from 13 on the window is split in two halves that meet in the middle: the best
+ * subset has the largest reachable Delta at or below the score's peak or the smallest above it (the
+ * appendix's two-probe rule), found by binary searches over the sorted subset sums of one half, per
+ * subset size.  That rule needs a score that is strictly monotone on both sides of its peak: Eq. 1
+ * with G >= 2, or Eq. 2 with H <= 16 and no segment slope within rounding distance of zero (checked
+ * by br_create); otherwise windows of up to 20 requests are enumerated and larger ones refused.
+ * Device pointers; asynchronous on batch.stream; BR_EINVAL for null pointers, R outside [1, 32], or
+ * R > 20 without the two-probe rule.
  */
 int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *win, int32_t R,
                    const int64_t *margins, const int32_t *lim, uint32_t *best_mask, double *best_F);

@@ -24,6 +24,7 @@ struct br_ctx {
     int threads_small;        // ... for batches of a few instances (latency path)
     int inst_per_block;       // single-warp instances per thread block
     bool small_ok;            // the fleet shape fits br_small_kernel
+    bool two_probe_ok;        // both sides of the score's peak are strictly monotone up to Delta = 32 s_max
     size_t smem;
     // latency path
     cudaGraph_t graph;
@@ -153,7 +154,8 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
         if (e != cudaSuccess) return cuda_fail(e, "br_step launch");
         return BR_OK;
     }
-    const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles) ? (tpi == 32 ? 2 : 1) : 0;
+    const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles && !ctx->base.big_window)
+                         ? (tpi == 32 ? 2 : 1) : 0;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
     // single-warp instances are packed several to a block
     // instances are packed several to a block: single-warp ones always, wider ones only in full
@@ -298,15 +300,23 @@ int br_create(int32_t G, int32_t H, const br_params *params, br_ctx **out)
             }
             const double err = 4.0 * (H + 5) * 1.1102230246251565e-16 * (a.aD + p.beta * D) * (double)p.s_max;
             a.peak_ok = (min_abs > err && min_abs > 1e-9) ? 1 : 0;
+            // the same for subsets of up to 32 requests (Delta <= 32 s_max): the two-probe rule of the
+            // large-window solvers
+            ctx->two_probe_ok = min_abs > 32.0 * err && min_abs > 1e-9;
         }
     } else {
         a.d[0] = 1.0; a.aD = 1.0; a.beta = (double)G; a.peak_ok = 0;
+        ctx->two_probe_ok = G >= 2;            // Eq. 1 falls with slope -(G - 1) beyond the margin
     }
-    ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words, p.term_mode == 3);
+    // Stage-2 windows beyond five requests are solved by meeting in the middle, which rests on the
+    // two-probe rule
+    a.big_window = p.R_max > br::kRegWin ? 1 : 0;
+    if (a.big_window && !ctx->two_probe_ok) { delete ctx; return BR_EINVAL; }
+    ctx->smem = br::step_smem_bytes(G, H, p.B, p.W, a.occ_words, p.term_mode == 3, a.big_window != 0);
     if (ctx->smem > 227 * 1024) { delete ctx; return BR_EINVAL; }      // one instance must fit a thread block's shared memory
     // br_small_kernel: Eq. 1, one worker per lane, one occupancy word, at most 512 waiting requests,
     // arrivals served by one Philox call, and negative queue keys scoring below every waiting request
-    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode <= 1 &&
+    ctx->small_ok = p.score_mode == 0 && G <= 32 && p.B <= 64 && p.W <= 512 && p.term_mode <= 1 && p.R_max <= br::kRegWin &&
                     p.burst_every == 0 && (!p.arr_cdf || p.arr_len <= 64) &&
                     (long long)(G - 1) * p.s_max + 65536 < (1ll << (31 - wl));
     *out = ctx;
@@ -635,7 +645,13 @@ int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *w
     for (int h = 0; h <= BR_MAX_H; ++h) a.f.d[h] = ctx->base.d[h];
     a.R = R; a.first_instance = batch->first_instance;
     a.win = win; a.m = margins; a.lim = lim; a.best_mask = best_mask; a.best_F = best_F;
-    br::br_subset_kernel<<<batch->n_instances, 256, 0, (cudaStream_t)batch->stream>>>(a);
+    // windows of 13 requests and more meet in the middle when the two-probe rule holds; without it
+    // only enumeration is exact, which stops at 20 requests
+    if (R > br::kSubsetMaxEnum && !ctx->two_probe_ok) return BR_EINVAL;
+    if (R > 12 && ctx->two_probe_ok)
+        br::br_subset_mitm_kernel<<<batch->n_instances, 256, 0, (cudaStream_t)batch->stream>>>(a);
+    else
+        br::br_subset_kernel<<<batch->n_instances, 256, 0, (cudaStream_t)batch->stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "br_best_subset launch");
     return BR_OK;

@@ -18,6 +18,7 @@
 // projection of BR-H streams the per-request state.
 #pragma once
 #include "br_device.cuh"
+#include "br_mitm.cuh"
 #include "../../include/br.h"
 
 namespace br {
@@ -40,6 +41,7 @@ struct StepArgs {
     int32_t burst_every, burst_size;
     double aD, beta;
     int32_t peak_ok;            // Eq. 2: every slope alpha D - beta sum_{h in P} d_h is clearly off zero (br_create)
+    int32_t big_window;         // R_max > 5: Stage 2 solves its window by meeting in the middle
     double d[BR_MAX_H + 1];
     int32_t N, first_instance, n_steps;
     int32_t tpi, smem_per_inst;  // threads and shared-memory bytes per instance
@@ -52,7 +54,8 @@ struct StepArgs {
 };
 
 // shared-memory footprint of one instance (bytes), mirrored by the host
-__host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words, bool lifetimes = false)
+__host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, int occ_words, bool lifetimes = false,
+                                                  bool big_window = false)
 {
     size_t n = 0;
     n += 4 * (size_t)W * 2;                      // q_key, q_id
@@ -65,6 +68,8 @@ __host__ __device__ inline size_t step_smem_bytes(int G, int H, int B, int W, in
     if (H > 0) n += 2 * (size_t)G * B;           // refresh_list
     n = (n + 15) & ~(size_t)15;
     if (lifetimes) n += 4 * (size_t)W;           // q_o (output lengths of the waiting requests)
+    n = (n + 15) & ~(size_t)15;
+    if (big_window) n += 8 * (size_t)(1 << 8) + 4 * 16 + 4 * 16;   // sorted half-window subsets, class offsets, window keys
     return (n + 15) & ~(size_t)15;
 }
 
@@ -169,6 +174,8 @@ __device__ __forceinline__ void draw_ending(const uint32_t *__restrict__ cdf, in
     }
 }
 
+constexpr int kRegWin = 5;      // Stage-2 windows of up to five requests are scored one subset per lane
+constexpr int kBigWinLow = 8;   // larger windows (up to BR_MAX_RMAX = 16): subsets of the low eight entries are sorted
 constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
@@ -219,6 +226,11 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     unsigned short *refresh_list = reinterpret_cast<unsigned short *>(scal + 16);   // [A] (H > 0 only)
     // output lengths of the waiting requests (term_mode 3 only), behind everything else
     int *q_o = reinterpret_cast<int *>(smem_raw + ((step_smem_bytes(G, H, B, W, OW) + 15) & ~(size_t)15));
+    // large Stage-2 windows: sorted subsets of the low half, class offsets, the window's keys
+    unsigned long long *bw_keys = reinterpret_cast<unsigned long long *>(
+        smem_raw + step_smem_bytes(G, H, B, W, OW, !LEAN && a.term_mode == 3));
+    int *bw_off = reinterpret_cast<int *>(bw_keys + (1 << kBigWinLow));
+    int *bw_win = bw_off + 16;
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
     //       [6] requests that ended this step and were not prefetched, [7] prefetched ones,
@@ -653,7 +665,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             int wt0 = 0, wt1 = 0, wt2 = 0, wt3 = 0, wt4 = 0;
             bool w_built = false, w_trunc = false;
             constexpr bool w_keep = FP;
-            int gw[BR_MAX_RMAX] = {0, 0, 0, 0, 0};
+            int gw[kRegWin] = {0, 0, 0, 0, 0};
             bool gw_valid = false;
 
             // argmax_i F_g({i}) over all waiting requests, earliest arrival on ties.
@@ -795,7 +807,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         Mh[h] = max(Mh[h], __shfl_sync(kFull, mine, src));
                     }
                 }
-                if (!w_keep && qk >= gw[BR_MAX_RMAX - 1]) gw_valid = false;   // one of the cached largest keys leaves
+                if (!w_keep && qk >= gw[kRegWin - 1]) gw_valid = false;   // one of the cached largest keys leaves
                 if (w_keep && w_built && lane == (pos & 31)) {
                     if (wt0 == qk) { wt0 = wt1; wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
                     else if (wt1 == qk) { wt1 = wt2; wt2 = wt3; wt3 = wt4; wt4 = 0; }
@@ -856,8 +868,106 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int g = (int)mg;
                     load_margins(g);
 
+                    if (!LEAN && a.big_window) {
+                        // ---- windows of 6 to 16 requests (Appendix "Bit-set subset selection") ----
+                        // the R_max largest keys, one warp maximum per entry (keys are distinct)
+                        const int R = min(a.R_max, n_left);
+                        int thr = 0x7FFFFFFF;
+                        for (int r = 0; r < R; ++r) {
+                            int best = 0;
+#pragma unroll 4
+                            for (int t = 0; t < n_tiles; ++t) {
+                                const int idx = (t << 5) + lane;
+                                const int x = idx < n_w ? q_key[idx] : 0;
+                                if (x < thr) best = max(best, x);
+                            }
+                            thr = __reduce_max_sync(kFull, best);
+                            if (lane == 0) bw_win[r] = thr;
+                        }
+                        __syncwarp();
+                        // prompt lengths of the window in shared memory (reusing the key slots' upper half is
+                        // not needed: lengths are recomputed from the keys)
+                        const int lim = min(mc, R);
+                        const int ra = min(kBigWinLow, (R + 1) / 2), rb = R - ra;
+                        // sorted subsets of the low entries (as prompt lengths)
+                        {
+                            const int n = 1 << ra;
+                            for (int m = lane; m < n; m += 32) {
+                                int sum = 0;
+                                for (int j = 0; j < ra; ++j) if ((m >> j) & 1) sum += bw_win[j] >> WL;
+                                bw_keys[m] = ((unsigned long long)__popc(m) << 56) | ((unsigned long long)(unsigned)sum << 16) | (unsigned)m;
+                            }
+                            __syncwarp();
+                            for (int k2 = 2; k2 <= n; k2 <<= 1) {
+                                for (int j = k2 >> 1; j > 0; j >>= 1) {
+                                    for (int i = lane; i < n; i += 32) {
+                                        const int p = i ^ j;
+                                        if (p > i) {
+                                            const unsigned long long x = bw_keys[i], y = bw_keys[p];
+                                            const bool up = (i & k2) == 0;
+                                            if ((x > y) == up) { bw_keys[i] = y; bw_keys[p] = x; }
+                                        }
+                                    }
+                                    __syncwarp();
+                                }
+                            }
+                            if (lane == 0) {
+                                int off = 0, binom = 1;
+                                for (int c = 0; c <= ra; ++c) { bw_off[c] = off; off += binom; binom = binom * (ra - c) / (c + 1); }
+                                bw_off[ra + 1] = off;
+                            }
+                            __syncwarp();
+                        }
+                        // the peak of the score in Delta
+                        int peak;
+                        if (!FP) {
+                            peak = sc.mi;
+                        } else {
+                            double mine = 0.0;
+#pragma unroll
+                            for (int h = 0; h <= HR; ++h) if (lane == h) mine = sc.md[h];
+                            double wsum = 0.0;
+#pragma unroll
+                            for (int h = 0; h <= HR; ++h) if (h <= H && sc.md[h] <= mine) wsum = __dadd_rn(wsum, a.d[h]);
+                            const bool past = lane <= H && !(a.aD > __dmul_rn(a.beta, wsum));
+                            peak = (int)__reduce_min_sync(kFull, past ? (unsigned)(int)mine : 0x7FFFFFFFu);
+                        }
+                        MitmBest b; b.lo_sum = -1; b.lo_mask = 0xFFFFFFFFu; b.hi_sum = 0x7FFFFFFF; b.hi_mask = 0xFFFFFFFFu;
+                        for (unsigned mh = lane; mh < (1u << rb); mh += 32) {
+                            const int ph = __popc(mh);
+                            if (ph > lim) continue;
+                            int sh = 0;
+                            for (unsigned t = mh; t; t &= t - 1) sh += bw_win[ra + __ffs(t) - 1] >> WL;
+                            mitm_probe(bw_keys, bw_off, ra, lim, peak, mh, sh, ph, b);
+                        }
+                        // warp reduction: largest sum at or below the peak, smallest above it, lowest mask among equals
+                        {
+                            const int ls = __reduce_max_sync(kFull, b.lo_sum);
+                            const unsigned lm = __reduce_min_sync(kFull, b.lo_sum == ls ? b.lo_mask : 0xFFFFFFFFu);
+                            const int hs = __reduce_min_sync(kFull, b.hi_sum);
+                            const unsigned hm = __reduce_min_sync(kFull, b.hi_sum == hs ? b.hi_mask : 0xFFFFFFFFu);
+                            b.lo_sum = ls; b.lo_mask = lm; b.hi_sum = hs; b.hi_mask = hm;
+                        }
+                        long long bk = kNoKey; unsigned bmask = 0u;
+                        if (b.lo_sum >= 0) { bk = sc.key(a, b.lo_sum); bmask = b.lo_mask; }
+                        if (b.hi_sum != 0x7FFFFFFF) {
+                            const long long k2 = sc.key(a, b.hi_sum);
+                            if (k2 > bk || (k2 == bk && b.hi_mask < bmask)) { bk = k2; bmask = b.hi_mask; }
+                        }
+                        if (bk == kNoKey) { status |= BR_ST_ITER_CAP; break; }
+                        if (bk <= 0) {
+                            const int qk = best_single();                   // starvation guard
+                            if (qk <= 0) break;
+                            commit(qk, g);
+                        } else {
+                            for (int r = 0; r < R; ++r)
+                                if ((bmask >> r) & 1u) commit(bw_win[r], g);
+                        }
+                        continue;
+                    }
+
                     // window: the R_max largest waiting requests, earliest first on ties
-                    int win[BR_MAX_RMAX];
+                    int win[kRegWin];
                     int nwin = 0;
                     if (!w_keep) {
                         // Eq. 1 kernels cache the five largest keys of the queue; the cache stays valid
@@ -876,7 +986,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                                 t4 = max(t4, x);
                             }
 #pragma unroll
-                            for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                            for (int r = 0; r < kRegWin; ++r) {
                                 const int m = __reduce_max_sync(kFull, t0);
                                 gw[r] = m;
                                 if (t0 == m) { t0 = t1; t1 = t2; t2 = t3; t3 = t4; t4 = 0; }
@@ -884,7 +994,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                             gw_valid = true;
                         }
 #pragma unroll
-                        for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                        for (int r = 0; r < kRegWin; ++r) {
                             win[r] = (r < a.R_max && r < n_left) ? gw[r] : 0;
                             if (win[r] > 0) nwin = r + 1;
                         }
@@ -916,7 +1026,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                             bool dry = false;
                             nwin = 0;
 #pragma unroll
-                            for (int r = 0; r < BR_MAX_RMAX; ++r) {
+                            for (int r = 0; r < kRegWin; ++r) {
                                 win[r] = 0;
                                 if (r < a.R_max && r < n_left) {
                                     dry = dry || (h0 == 0 && w_trunc);
@@ -936,7 +1046,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     if (lane >= 1 && lane < (1 << nwin) && __popc(lane) <= lim) {
                         int delta = 0;
 #pragma unroll
-                        for (int r = 0; r < BR_MAX_RMAX; ++r)
+                        for (int r = 0; r < kRegWin; ++r)
                             if ((lane >> r) & 1) delta += win[r] >> WL;
                         fk = sc.key(a, delta);
                     }
@@ -957,7 +1067,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         commit(qk, g);
                     } else {
 #pragma unroll
-                        for (int r = 0; r < BR_MAX_RMAX; ++r)
+                        for (int r = 0; r < kRegWin; ++r)
                             if ((best_mask >> r) & 1) commit(win[r], g);
                     }
                 }

@@ -57,7 +57,7 @@ def test_create_validates_sizes_and_ranges():
     assert L.br_destroy(None) == BR_OK
     for G, H, kw in [(0, 0, {}), (65, 0, {}), (32, 81, {}), (32, -1, {}), (32, 0, dict(B=12)),
                      (32, 0, dict(B=264)), (32, 0, dict(W=6)), (32, 0, dict(W=8192)),
-                     (32, 0, dict(R_max=6)), (32, 4, dict(score_mode=0)), (32, 0, dict(term_mode=2)),
+                     (32, 0, dict(R_max=17)), (32, 4, dict(score_mode=0)), (32, 0, dict(term_mode=2)),
                      (32, 0, dict(term_mode=4)), (32, 4, dict(pred_mode=1)), (32, 0, dict(term_mode=3, pred_mode=1)), (32, 0, dict(term_cdf=None)), (32, 4, dict(gamma=0.0)), (32, 4, dict(gamma=1.5)),
                      (32, 4, dict(alpha=-1.0)), (32, 0, dict(threads=48)), (32, 0, dict(threads=512)),
                      (32, 4, dict(delta_T=200))]:

@@ -261,3 +261,24 @@ def test_long_horizon_multi_step_and_random_shapes():
                              arrival=("const", float(rng.choice([1.0, 8.0]))), first_seed=7000 * case)
         run_parity(cfg, 2, 30, threads=int(rng.choice([0, 32, 128])), check_every=10,
                    launch_steps=int(rng.choice([1, 3])))
+
+
+@pytest.mark.parametrize("name,R_max,kw", [("c1", 6, {}), ("c1", 16, dict(S_greedy=1 << 20)), ("c2", 9, {}),
+                                           ("c2", 16, dict(gate=0.0, delta_T=1, S_greedy=1 << 20)),
+                                           ("c4", 12, {}), ("c3", 7, dict(hazard=0.05))])
+def test_large_stage2_windows(name, R_max, kw):
+    """Windows of 6 to 16 requests: Stage 2 picks its subset by meeting in the middle."""
+    run_parity(wlm.get_config(name, R_max=R_max, **kw), 2, 60, check_every=10)
+
+
+def test_large_stage2_windows_random_shapes():
+    rng = np.random.default_rng(1616)
+    for case in range(8):
+        G = int(rng.integers(2, 65)); B = 8 * int(rng.integers(1, 9)); W = 4 * int(rng.integers(2, 100))
+        H = int(rng.choice([0, 0, 3, 8, 16]))
+        cfg = wlm.get_config("c2" if H else "c1", G=G, B=B, W=W, H=H, R_max=int(rng.integers(6, 17)),
+                             S_greedy=int(rng.choice([-1, 0, 1 << 20])), hazard=float(rng.choice([0.02, 0.2])),
+                             term_mode=1, init_active=int(rng.integers(0, B + 1)), init_queue=int(rng.integers(0, W + 1)),
+                             arrival=("const", float(rng.choice([2.0, 12.0]))), first_seed=3100 * case)
+        run_parity(cfg, 2, 30, threads=int(rng.choice([0, 32, 128])), check_every=10,
+                   launch_steps=int(rng.choice([1, 4])))
