@@ -157,7 +157,6 @@ int launch_step(br_ctx *ctx, const br_instance_batch *b, const br_worker_state *
     const int lean = (ctx->p.term_mode == 1 && !out->fscore && !out->phase_cycles && !ctx->base.big_window)
                          ? (tpi == 32 ? 2 : 1) : 0;
     step_kernel_t kern = pick_kernel(ctx->p.score_mode == 1, ctx->H, ctx->G, lean);
-    // single-warp instances are packed several to a block
     // instances are packed several to a block: single-warp ones always, wider ones only in full
     // blocks (their barriers are block barriers)
     int per_block = ctx->inst_per_block;

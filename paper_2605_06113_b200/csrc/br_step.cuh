@@ -174,9 +174,38 @@ __device__ __forceinline__ void draw_ending(const uint32_t *__restrict__ cdf, in
     }
 }
 
+// Loads of classifier output.  A row is read once, by one thread, at a scattered address; left to
+// itself the L2 fetches 128 bytes around a missing sector, of which a refresh uses 32 on average,
+// so the loads ask for the smallest fetch the instruction set offers (64 bytes).
+__device__ __forceinline__ float4 ld_row4(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.L2::64B.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+// a whole row of eight probabilities (32-byte aligned) as one 256-bit load
+__device__ __forceinline__ void ld_row8(const float *p, float *o)
+{
+    unsigned r[8];
+    asm volatile("ld.global.nc.L2::64B.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) : "l"(p));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = __uint_as_float(r[i]);
+}
+
+// Adds (val, 1) to the prediction bucket `key` (load sum in T, count in C) if key >= 0.  Plain
+// shared-memory atomics: combining the lanes of a warp that share a bucket first (match.any and a
+// masked reduction) measured 70 % slower than letting the atomics collide.
+__device__ __forceinline__ void bucket_add(unsigned *T, unsigned *C, int key, unsigned val, int lane)
+{
+    (void)lane;
+    if (key >= 0) { atomicAdd(&T[key], val); atomicAdd(&C[key], 1u); }
+}
+
 constexpr int kRegWin = 5;      // Stage-2 windows of up to five requests are scored one subset per lane
 constexpr int kBigWinLow = 8;   // larger windows (up to BR_MAX_RMAX = 16): subsets of the low eight entries are sorted
-constexpr int kUnroll = 2;      // slot quads in flight per thread in the BR-H streaming phase
+constexpr int kPassBUnroll = 2;  // classifier rows in flight per thread (4 and 8 measured the same)
+constexpr int kUnroll = 2;       // slot quads in flight per thread in the BR-H streaming phase (4 measured the same)
 constexpr int kEndList = 96;    // requests ending in one step that are fixed up as one batch
 
 // LEAN > 0: constant-hazard terminations and no optional outputs (score matrix, cycle counters);
@@ -199,6 +228,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     // Instance-wide barrier.  Single-warp instances that share a block may also be aligned with a
     // block barrier (a.block_sync): the warps then walk the same code at about the same time, which
     // pays off in instruction fetch although no data crosses between them.
+    // (Giving wider instances that share a block a named barrier each, so that one never waits for
+    // its neighbour, measured 3 % slower on the 1024-instance BR-H batch: instances that walk the
+    // phases together share instruction fetch and keep the memory phases aligned.)
     auto inst_sync = [&]() { if (NT == 32 && !a.block_sync) __syncwarp(); else __syncthreads(); };
     const int nwarps = LEAN == 2 ? 1 : (NT >> 5);
     const int term_mode = LEAN ? 1 : a.term_mode;
@@ -416,20 +448,20 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             // perfect lookahead: c_hat = min(r_i(k), H) with r_i(k) = act_end - k + 1 steps still to run
             const int A4 = A >> 2;
 #pragma unroll 2
-            for (int q4 = tid; q4 < A4; q4 += NT) {
-                const int4 bq = *reinterpret_cast<const int4 *>(g_base + 4 * q4);
-                const int4 eq = *reinterpret_cast<const int4 *>(g_end + 4 * q4);
+            for (int q0 = 0; q0 < A4; q0 += NT) {
+                const int q4 = q0 + tid;
+                const bool inr = q4 < A4;
+                const int4 bq = inr ? *reinterpret_cast<const int4 *>(g_base + 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
+                const int4 eq = inr ? *reinterpret_cast<const int4 *>(g_end + 4 * q4) : make_int4(0, 0, 0, 0);
                 const int bs4[4] = {bq.x, bq.y, bq.z, bq.w};
                 const int en4[4] = {eq.x, eq.y, eq.z, eq.w};
                 const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    if (bs4[j] != kEmpty) {
-                        int nh = en4[j] - k + 1;
-                        nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                        atomicAdd(&Lh_s[g * H1 + nh], (unsigned)(bs4[j] + k));
-                        atomicAdd(&Ch_s[g * H1 + nh], 1u);
-                    }
+                    const bool live = bs4[j] != kEmpty;
+                    int nh = en4[j] - k + 1;
+                    nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                    bucket_add(Lh_s, Ch_s, live ? g * H1 + nh : -1, live ? (unsigned)(bs4[j] + k) : 0u, lane);
                 }
             }
         } else if (HM > 0 && H > 0) {
@@ -451,109 +483,111 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const int bs4[4] = {bq[u].x, bq[u].y, bq[u].z, bq[u].w};
                     const float c04[4] = {cq[u].x, cq[u].y, cq[u].z, cq[u].w};
                     const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);      // slot / B
+                    // which of the four requests are due for a refresh; one list append per quad and warp
+                    bool due4[4]; float c4[4]; unsigned dm4[4];
+                    int n_due = 0;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const bool live = bs4[j] != kEmpty;
                         const int t = (k - (int)((kq[u] >> (8 * j)) & 0xFFu)) & 255;
-                        const float c = c04[j] - (float)t;
-                        const bool due = live && (t >= a.delta_T || c < a.c_floor);
-                        const unsigned dm = __ballot_sync(kFull, due);          // one list append per warp
-                        if (dm) {
-                            const int lead = __ffs(dm) - 1;
-                            int at = 0;
-                            if (lane == lead) at = atomicAdd(&scal[8], __popc(dm));
-                            at = __shfl_sync(kFull, at, lead);
-                            if (due) refresh_list[at + __popc(dm & ((1u << lane) - 1u))] = (unsigned short)(4 * q4 + j);
+                        c4[j] = c04[j] - (float)t;
+                        due4[j] = live && (t >= a.delta_T || c4[j] < a.c_floor);
+                        dm4[j] = __ballot_sync(kFull, due4[j]);
+                        n_due += __popc(dm4[j]);
+                    }
+                    if (n_due) {                                             // uniform over the warp
+                        int at = 0;
+                        if (lane == 0) at = atomicAdd(&scal[8], n_due);
+                        at = __shfl_sync(kFull, at, 0);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (due4[j]) refresh_list[at + __popc(dm4[j] & ((1u << lane) - 1u))] = (unsigned short)(4 * q4 + j);
+                            at += __popc(dm4[j]);
                         }
-                        if (live && !due) {
-                            int nh = (int)floorf(c);
-                            nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                            atomicAdd(&Lh_s[g * H1 + nh], (unsigned)(bs4[j] + k));
-                            atomicAdd(&Ch_s[g * H1 + nh], 1u);
-                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const bool settle = bs4[j] != kEmpty && !due4[j];
+                        int nh = (int)floorf(c4[j]);
+                        nh = nh < 0 ? 0 : (nh > H ? H : nh);
+                        bucket_add(Lh_s, Ch_s, settle ? g * H1 + nh : -1, settle ? (unsigned)(bs4[j] + k) : 0u, lane);
                     }
                 }
             }
             inst_sync();
             const int n_ref = scal[8];
-#pragma unroll 2
-            for (int e = tid; e < n_ref; e += NT) {
-                const int s0 = refresh_list[e];
-                const float *q = probs + (size_t)s0 * H;
-                if (SL) {
-                    // long classifier rows stay in memory: one pass for p_fin, one for c*
-                    double surv = 1.0, cs = 0.0;
-                    for (int h = 0; h < H; ++h) {
-                        cs = __dadd_rn(cs, surv);
-                        surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
+            // Pass B: the classifier row of every request on the list.  The loop runs the same number of
+            // rounds on every lane.
+#pragma unroll kPassBUnroll
+            for (int e0 = 0; e0 < n_ref; e0 += NT) {
+                const int e = e0 + tid;
+                int key = -1;
+                unsigned cur = 0u;
+                if (e < n_ref) {
+                    const int s0 = refresh_list[e];
+                    const float *q = probs + (size_t)s0 * H;
+                    double v = (double)H;                               // gate closed: the conservative anchor
+                    if (SL) {
+                        // long classifier rows stay in memory: p_fin and c* in one pass
+                        double surv = 1.0, cs = 0.0;
+                        for (int h = 0; h < H; ++h) {
+                            cs = __dadd_rn(cs, surv);
+                            surv = __dmul_rn(surv, __dsub_rn(1.0, (double)q[h]));
+                        }
+                        if (__dsub_rn(1.0, surv) >= (double)a.gate) v = cs;
+                    } else {
+                        float qv[HR > 0 ? HR : 1];
+                        if (HR == 8 && H == 8 && (reinterpret_cast<size_t>(probs) & 31) == 0) {
+                            ld_row8(q, qv);
+                        } else if ((H & 3) == 0) {
+#pragma unroll
+                            for (int h = 0; h < HR; h += 4) {
+                                if (h < H) {
+                                    const float4 qq = ld_row4(q + h);
+                                    qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int h = 0; h < HR; ++h) if (h < H) qv[h] = q[h];
+                        }
+                        // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
+                        // clearly below the gate the fp64 product cannot reach it and is not evaluated
+                        float qsum = 0.0f, qmin = 0.0f;
+#pragma unroll
+                        for (int h = 0; h < HR; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
+                        double p_fin = 0.0;
+                        if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
+                            double surv = 1.0;
+#pragma unroll
+                            for (int h = 0; h < HR; ++h)
+                                if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
+                            p_fin = __dsub_rn(1.0, surv);
+                        }
+                        if (p_fin >= (double)a.gate) {
+                            // gate open: E[min(r, H)] = sum_h prod_{j<h} (1 - q_j)
+                            double sv = 1.0, cs = 0.0;
+#pragma unroll
+                            for (int h = 0; h < HR; ++h) {
+                                if (h < H) {
+                                    cs = __dadd_rn(cs, sv);
+                                    sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
+                                }
+                            }
+                            v = cs;
+                        }
                     }
-                    double v = (double)H;
-                    if (__dsub_rn(1.0, surv) >= (double)a.gate) {
-                        v = cs;
-                        if (v < (double)a.c_floor) v = (double)a.c_floor;
-                        if (v > (double)H) v = (double)H;
-                    }
+                    if (v < (double)a.c_floor) v = (double)a.c_floor;   // clipped to [floor, H]
+                    if (v > (double)H) v = (double)H;
                     const float c = (float)v;
-                    const int cur = g_base[s0] + k;
+                    cur = (unsigned)(g_base[s0] + k);
                     g_chat0[s0] = c;
                     g_kref[s0] = (uint8_t)(k & 255);
                     int nh = (int)floorf(c);
                     nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                    const int g = (int)__umulhi((unsigned)s0, a.magic_B);
-                    atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
-                    atomicAdd(&Ch_s[g * H1 + nh], 1u);
-                    continue;
+                    key = (int)__umulhi((unsigned)s0, a.magic_B) * H1 + nh;
                 }
-                float qv[HR > 0 ? HR : 1];
-                if ((H & 3) == 0) {
-#pragma unroll
-                    for (int h = 0; h < HR; h += 4) {
-                        if (h < H) {
-                            const float4 qq = *reinterpret_cast<const float4 *>(q + h);
-                            qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int h = 0; h < HR; ++h) if (h < H) qv[h] = q[h];
-                }
-                const int cur = g_base[s0] + k;
-                // p_fin = 1 - prod (1 - q_h) <= sum q_h for probabilities: when the fp32 sum is
-                // clearly below the gate the fp64 product cannot reach it and is not evaluated
-                float qsum = 0.0f, qmin = 0.0f;
-#pragma unroll
-                for (int h = 0; h < HR; ++h) if (h < H) { qsum += qv[h]; qmin = fminf(qmin, qv[h]); }
-                double p_fin = 0.0;
-                if (!(qmin >= 0.0f && qsum * 1.0001f < a.gate)) {
-                    double surv = 1.0;
-#pragma unroll
-                    for (int h = 0; h < HR; ++h)
-                        if (h < H) surv = __dmul_rn(surv, __dsub_rn(1.0, (double)qv[h]));
-                    p_fin = __dsub_rn(1.0, surv);
-                }
-                double v = (double)H;
-                if (p_fin >= (double)a.gate) {
-                    // gate open: E[min(r, H)] = sum_h prod_{j<h} (1 - q_j), clipped to [floor, H]
-                    double sv = 1.0, cs = 0.0;
-#pragma unroll
-                    for (int h = 0; h < HR; ++h) {
-                        if (h < H) {
-                            cs = __dadd_rn(cs, sv);
-                            sv = __dmul_rn(sv, __dsub_rn(1.0, (double)qv[h]));
-                        }
-                    }
-                    v = cs;
-                    if (v < (double)a.c_floor) v = (double)a.c_floor;
-                    if (v > (double)H) v = (double)H;
-                }
-                const float c = (float)v;
-                g_chat0[s0] = c;
-                g_kref[s0] = (uint8_t)(k & 255);
-                int nh = (int)floorf(c);
-                nh = nh < 0 ? 0 : (nh > H ? H : nh);
-                const int g = (int)__umulhi((unsigned)s0, a.magic_B);
-                atomicAdd(&Lh_s[g * H1 + nh], (unsigned)cur);
-                atomicAdd(&Ch_s[g * H1 + nh], 1u);
+                bucket_add(Lh_s, Ch_s, key, cur, lane);
             }
         }
         inst_sync();                                              // B1
@@ -1105,54 +1139,74 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         inst_sync();                                              // B2: admissions visible
 
         // ============ queue compaction and assignments (warp 0) ============
+        // A lane owns four consecutive positions of every group of 128 (16-byte accesses to the keys,
+        // the ids and the assignment row); an entry's new position is the count of kept entries before it.
         if (warp == 0) {
             int32_t *assign = a.assign_out + orow * W;
             int run = 0;
             const int n_before = n_w;          // queue length after ARRIVE
-#pragma unroll 2
-            for (int i0 = 0; i0 < W; i0 += 32) {
-                const int i = i0 + lane;
-                const bool inq = i < n_before;
-                const int qk = inq ? q_key[i] : 0;
-                const unsigned id = inq ? q_id[i] : 0u;
-                const int qo = (life && inq) ? q_o[i] : 0;
-                const bool gone = inq && qk < 0;
-                const bool keep = inq && qk > 0;
-                const unsigned bal = __ballot_sync(kFull, keep);
-                const int dst = run + __popc(bal & ((1u << lane) - 1u));
-                const int sa = qk & 0x7FFFFFFF;
-                if (i < W) assign[i] = (gone && sa < A) ? sa : -1;
-                if (have_pre && gone && sa < A) {
-                    // a request admitted at this step may also end at it
-                    const int g = (int)__umulhi((unsigned)sa, a.magic_B), slot = sa - g * B;
-                    if ((fin_w[g * OW + (slot >> 6)] >> (slot & 63)) & 1ull) {
-                        atomicOr(&end_mask[g * OW + (slot >> 6)], 1ull << (slot & 63));
-                        const int at = atomicAdd(&scal[6], 1);
-                        if (at < kEndList) {
-                            end_list[at] = (unsigned short)sa;
-                        } else {
-                            atomicAdd(&sub_load[g], (unsigned)(g_base[sa] + k));
-                            g_base[sa] = kEmpty;
+            const unsigned lt = (1u << lane) - 1u;
+#pragma unroll 1
+            for (int i0 = 0; i0 < W; i0 += 128) {
+                const int p0 = i0 + lane * 4;
+                if (i0 >= n_before) {
+                    // the rest of the row is beyond the queue: only assignments remain
+                    if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(-1, -1, -1, -1);
+                    continue;
+                }
+                int4 kk = make_int4(0, 0, 0, 0); uint4 ii = make_uint4(0u, 0u, 0u, 0u); int4 oo = make_int4(0, 0, 0, 0);
+                if (p0 < W) {
+                    kk = *reinterpret_cast<const int4 *>(q_key + p0);
+                    ii = *reinterpret_cast<const uint4 *>(q_id + p0);
+                    if (life) oo = *reinterpret_cast<const int4 *>(q_o + p0);
+                }
+                int ke[4] = {kk.x, kk.y, kk.z, kk.w};
+                const unsigned idv[4] = {ii.x, ii.y, ii.z, ii.w};
+                const int ov[4] = {oo.x, oo.y, oo.z, oo.w};
+                int as[4];
+                int below = run, total = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (p0 + j >= n_before) ke[j] = 0;                  // beyond the queue
+                    const unsigned bal = __ballot_sync(kFull, ke[j] > 0);
+                    below += __popc(bal & lt);
+                    total += __popc(bal);
+                    const int sa = ke[j] & 0x7FFFFFFF;
+                    const bool gone = ke[j] < 0 && sa < A;
+                    as[j] = gone ? sa : -1;
+                    if (have_pre && gone) {
+                        // a request admitted at this step may also end at it
+                        const int g = (int)__umulhi((unsigned)sa, a.magic_B), slot = sa - g * B;
+                        if ((fin_w[g * OW + (slot >> 6)] >> (slot & 63)) & 1ull) {
+                            atomicOr(&end_mask[g * OW + (slot >> 6)], 1ull << (slot & 63));
+                            const int at = atomicAdd(&scal[6], 1);
+                            if (at < kEndList) {
+                                end_list[at] = (unsigned short)sa;
+                            } else {
+                                atomicAdd(&sub_load[g], (unsigned)(g_base[sa] + k));
+                                g_base[sa] = kEmpty;
+                            }
                         }
                     }
                 }
-                __syncwarp();
-                if (keep) {
-                    const int s = qk >> WL;
-                    if (dst != i) { q_key[dst] = (s << WL) | (int)(posmask - (unsigned)dst); q_id[dst] = id; }
-                    if (dst != i || i >= n_w_old) { g_qs[dst] = s; g_qid[dst] = id; }
-                    if (life) {
-                        if (dst != i) q_o[dst] = qo;
-                        if (dst != i || i >= n_w_old) g_qo[dst] = qo;
+                if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(as[0], as[1], as[2], as[3]);
+                __syncwarp();                                           // the group is read before any of it is overwritten
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (ke[j] > 0) {
+                        const int i = p0 + j, dst = below;
+                        const int sv = ke[j] >> WL;
+                        if (dst != i) { q_key[dst] = (sv << WL) | (int)(posmask - (unsigned)dst); q_id[dst] = idv[j]; }
+                        if (dst != i || i >= n_w_old) { g_qs[dst] = sv; g_qid[dst] = idv[j]; }
+                        if (life) {
+                            if (dst != i) q_o[dst] = ov[j];
+                            if (dst != i || i >= n_w_old) g_qo[dst] = ov[j];
+                        }
+                        ++below;
                     }
                 }
                 __syncwarp();
-                run += __popc(bal);
-                if (i0 + 32 >= n_before) {
-                    // the rest of the row is beyond the queue: only assignments remain
-                    for (int j = i0 + 32 + lane; j < W; j += 32) assign[j] = -1;
-                    break;
-                }
+                run += total;
             }
         }
         n_w = scal[0];
