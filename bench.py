@@ -412,6 +412,7 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
                         probs_ring=probs_ring, spl=spl, start_steps=starts)
     starts = list(sets.start_steps)
+    launches_before = sum(st // spl for st in starts) + warmup + prime      # before the first timed call
     for _ in range(warmup):
         sets.step()
     torch.cuda.synchronize()
@@ -439,6 +440,7 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
     us_per_launch = 1e3 * ms / launches
     return dict(ms=ms, ms_per_launch=ms / launches, us_per_launch=us_per_launch, n_sets=n_sets, N=N, spl=spl,
+                launches_before_timed=launches_before,
                 trajectory=f"sets start at decode steps {starts} of {cfg.steps} and advance {span} steps per repeat",
                 repeats_ms=[float(x) for x in reps], abytes_per_launch=abytes,
                 achieved=abytes / (us_per_launch * 1e-6) / 1e9, bad=bad, clocks=clocks, threads=tpi,
@@ -520,7 +522,7 @@ def run_ours(args):
                    "timing": f"median of {args.repeats} repeats of the {args.steps}-call region (CUDA events; "
                              f"before each repeat the sets return to their starting snapshots and one untimed "
                              f"call per set runs)",
-                   "trajectory": m["trajectory"],
+                   "trajectory": m["trajectory"], "launches_before_timed": m["launches_before_timed"],
                    "l2": f"{m['n_sets']} instance sets stepped in rotation: data touched between two visits of a "
                          f"set exceeds the 126 MB L2; no instance runs past the configuration's {cfg.steps} steps",
                    "threads_per_instance": m["threads"]},

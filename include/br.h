@@ -217,11 +217,13 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *w
  * Otherwise arguments, results and status codes are those of br_step_host.
  *
  * The first call on each device looks up the array's device address (a CUDA runtime query
- * made with that device current; no allocation).  Make that first call outside any stream
- * capture.  All calls on a device share the one array, which still holds the previous
- * call's data: inputs are overwritten by the copies of this call and the output blocks are
- * cleared first, but two calls that overlap on the GPU (different streams, or different host
- * threads) race on it -- serialise them.  The call returns after synchronising the stream.
+ * made with that device current; no allocation) and keeps it for later calls.  Make that first
+ * call before any stream capture begins on the thread; the entry point itself ends with a stream
+ * synchronisation and therefore never belongs inside a capture.  All calls on a device share the
+ * one array, which still holds the previous call's data: inputs are overwritten by the copies of
+ * this call and the output blocks are cleared first, but two calls that overlap on the GPU
+ * (different streams, or different host threads) race on it -- serialise them.  If a CUDA call
+ * fails after copies have been queued, the stream is drained before the error is returned.
  */
 #define BR_STATIC_STAGE_BYTES (8u << 20)
 int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *worker_state,
@@ -266,7 +268,7 @@ int br_best_subset(br_ctx *ctx, const br_instance_batch *batch, const int32_t *w
  * routed one at a time in arrival order: request i goes to argmax_g F_g(s_i) (Eq. 1 with the
  * context's coefficients, lowest g on ties) over the workers with inflight[g] < inflight_cap[g],
  * where the margins m_g = M - L_g come from the virtual loads virtual_load [N][G] (running plus
- * dispatched-but-not-yet-running requests).  The chosen worker's virtual load grows by s_i and its
+ * requests that were dispatched and have not started yet).  The chosen worker's virtual load grows by s_i and its
  * inflight count by one before the next request is scored.  worker_out [N][n_requests] receives
  * the worker, -1 when every worker is at its cap; virtual_load and inflight are updated in place.
  * Device pointers, asynchronous on batch.stream.

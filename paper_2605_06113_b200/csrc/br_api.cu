@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <atomic>
 #include <new>
 
 #include "br_step.cuh"
@@ -51,6 +52,18 @@ int cuda_fail(cudaError_t e, const char *what)
     do {                                                   \
         cudaError_t e__ = (call);                          \
         if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+// For calls made after work has been queued on `stream`: on failure the stream is drained first,
+// so that no copy still reads or writes the caller's buffers (or the shared staging) when the error
+// is reported.
+#define BR_CUDA_DRAIN(call, stream)                        \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) {                          \
+            cudaStreamSynchronize(stream);                 \
+            return cuda_fail(e__, #call);                  \
+        }                                                  \
     } while (0)
 
 inline bool misaligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
@@ -473,6 +486,13 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         for (int i = 0; i < 2 * 8 + 2; ++i) BR_CUDA(cudaEventCreateWithFlags(&ctx->pipe_ev[i], cudaEventDisableTiming));
         ctx->pipe_ready = true;
     }
+    // once copies are queued an error drains the device before it is reported (the copies use the
+    // caller's buffers and up to three streams)
+#define BR_HOST_STEP(call)                                            \
+    do {                                                              \
+        cudaError_t e__ = (call);                                     \
+        if (e__ != cudaSuccess) { cudaDeviceSynchronize(); return cuda_fail(e__, #call); } \
+    } while (0)
     cudaStream_t s_in = st, s_k = st, s_out = st;
     if (n_chunks > 1) {
         s_in = ctx->pipe[0]; s_k = ctx->pipe[1]; s_out = ctx->pipe[2];
@@ -484,13 +504,13 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
     if (n_chunks > 1)
         for (Blk &b : blks)
             if (b.bytes && b.in && b.bytes < kBig)
-                BR_CUDA(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, s_in));
+                BR_HOST_STEP(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, s_in));
     for (int c = 0; c < n_chunks; ++c) {
         const size_t i0 = N * (size_t)c / n_chunks, i1 = N * (size_t)(c + 1) / n_chunks;
         for (Blk &b : blks) {
             if (!b.bytes || !b.in || (n_chunks > 1 && b.bytes < kBig)) continue;
             const size_t row = b.bytes / N;
-            BR_CUDA(cudaMemcpyAsync((char *)*b.dev + i0 * row, (const char *)b.host + i0 * row, (i1 - i0) * row,
+            BR_HOST_STEP(cudaMemcpyAsync((char *)*b.dev + i0 * row, (const char *)b.host + i0 * row, (i1 - i0) * row,
                                     cudaMemcpyHostToDevice, s_in));
         }
         if (n_chunks > 1) {
@@ -500,7 +520,7 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         br_instance_batch cb = db;
         cb.first_instance = (int32_t)i0; cb.n_instances = (int32_t)(i1 - i0);
         rc = launch_step(ctx, &cb, &dws, &dwq, d_probs, d_assign, &dout, s_k);   // rows are addressed through first_instance
-        if (rc != BR_OK) return rc;
+        if (rc != BR_OK) { cudaDeviceSynchronize(); return rc; }
         if (n_chunks > 1) {
             BR_CUDA(cudaEventRecord(ctx->pipe_ev[8 + c], s_k));
             BR_CUDA(cudaStreamWaitEvent(s_out, ctx->pipe_ev[8 + c], 0));
@@ -508,19 +528,20 @@ int br_step_host(br_ctx *ctx, const br_instance_batch *batch, br_worker_state *h
         for (Blk &b : blks) {
             if (!b.bytes || !b.out || (n_chunks > 1 && b.bytes < kBig)) continue;
             const size_t row = b.bytes / N;
-            BR_CUDA(cudaMemcpyAsync((char *)b.host + i0 * row, (const char *)*b.dev + i0 * row, (i1 - i0) * row,
+            BR_HOST_STEP(cudaMemcpyAsync((char *)b.host + i0 * row, (const char *)*b.dev + i0 * row, (i1 - i0) * row,
                                     cudaMemcpyDeviceToHost, s_out));
         }
     }
     if (n_chunks > 1)
         for (Blk &b : blks)                              // s_out has waited for the last kernel
             if (b.bytes && b.out && b.bytes < kBig)
-                BR_CUDA(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, s_out));
+                BR_HOST_STEP(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, s_out));
     if (n_chunks > 1) {
         BR_CUDA(cudaEventRecord(ctx->pipe_ev[17], s_out));
         BR_CUDA(cudaStreamWaitEvent(st, ctx->pipe_ev[17], 0));
     }
     BR_CUDA(cudaStreamSynchronize(st));
+#undef BR_HOST_STEP
     if (h2d_bytes) *h2d_bytes = up;
     if (d2h_bytes) *d2h_bytes = down;
     return BR_OK;
@@ -534,7 +555,10 @@ static __device__ __align__(256) unsigned char g_static_stage[BR_STATIC_STAGE_BY
 
 namespace {
 constexpr int kMaxDevices = 64;
-void *g_static_stage_ptr[kMaxDevices];      // device address of g_static_stage, per device
+// device address of g_static_stage, per device (looked up once; two threads that race on the first
+// call both store the same address).  cudaDeviceReset invalidates it: the library does not support
+// being used across a device reset.
+std::atomic<void *> g_static_stage_ptr[kMaxDevices];
 
 // In host code `g_static_stage` is only a handle; the address a kernel or a copy can use
 // has to be asked for, once per device, with that device current.
@@ -544,13 +568,13 @@ int static_stage_address(void **out)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
     if (dev < 0 || dev >= kMaxDevices) return BR_EINVAL;
-    if (!g_static_stage_ptr[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_static_stage_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress((void **)&ptr, g_static_stage);
         if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(g_static_stage)");
-        g_static_stage_ptr[dev] = ptr;
+        g_static_stage_ptr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_static_stage_ptr[dev];
+    *out = ptr;
     return BR_OK;
 }
 }  // namespace
@@ -584,18 +608,17 @@ int br_step_host_static(br_ctx *ctx, const br_instance_batch *batch, br_worker_s
         *b.dev = (char *)stage + off;
         if (!b.in) { if (!out_end) out_begin = off; out_end = off + ((b.bytes + 255) & ~(size_t)255); }
         off += (b.bytes + 255) & ~(size_t)255;
-        if (b.in) { BR_CUDA(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, st)); up += (int64_t)b.bytes; }
+        if (b.in) { BR_CUDA_DRAIN(cudaMemcpyAsync(*b.dev, b.host, b.bytes, cudaMemcpyHostToDevice, st), st); up += (int64_t)b.bytes; }
     }
     // the buffer still holds the previous call's results: the output blocks start from zero
-    if (out_end > out_begin) BR_CUDA(cudaMemsetAsync((char *)stage + out_begin, 0, out_end - out_begin, st));
+    if (out_end > out_begin) BR_CUDA_DRAIN(cudaMemsetAsync((char *)stage + out_begin, 0, out_end - out_begin, st), st);
     br_instance_batch db = *batch; db.n_steps = 1;
     rc = check_step_args(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout);
-    if (rc != BR_OK) return rc;
-    rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
-    if (rc != BR_OK) return rc;
+    if (rc == BR_OK) rc = launch_step(ctx, &db, &dws, &dwq, d_probs, d_assign, &dout, st);
+    if (rc != BR_OK) { cudaStreamSynchronize(st); return rc; }
     for (Blk &b : blks) {
         if (!b.bytes || !b.out) continue;
-        BR_CUDA(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, st));
+        BR_CUDA_DRAIN(cudaMemcpyAsync(b.host, *b.dev, b.bytes, cudaMemcpyDeviceToHost, st), st);
         down += (int64_t)b.bytes;
     }
     BR_CUDA(cudaStreamSynchronize(st));

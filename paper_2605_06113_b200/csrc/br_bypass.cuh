@@ -1,7 +1,7 @@
 // Pool-bypass dispatch for BR-0 (Appendix "Pool-bypass deployment path for BR-0"): requests are
 // routed one at a time, in arrival order, each to argmax_g F_g(s) = alpha s - beta (s - m_g)_+ over
 // the workers whose inflight count is below its cap, with m_g = M - L_g taken from *virtual*
-// loads (running plus dispatched-but-not-yet-running requests); the chosen worker's virtual load
+// loads (running requests plus those dispatched and not started yet); the chosen worker's virtual load
 // and inflight count grow at once, so the next request sees them.  One warp per instance, lane g
 // holds worker g (and g + 32): the chain over requests is sequential, the arg-max over workers a
 // warp reduction with lowest-g tie-break.

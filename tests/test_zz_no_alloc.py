@@ -7,6 +7,7 @@ row (the second call reuses the built-in staging array with the first call's dat
 Collected last on purpose: a failure here cannot hide the result of any other test."""
 import numpy as np
 import pytest
+import torch
 
 from paper_2605_06113_b200 import workload as wlm
 from paper_2605_06113_b200.binding import BR_ELIMIT, BrError, Router, STATIC_STAGE_BYTES
@@ -27,10 +28,15 @@ def test_static_staging_matches_allocating_entry_point(name, n_inst):
     r = Router(wl, device="cuda:0")
     st_a, out_a = _host_buffers(wl, r, n_inst)      # br_step_host (allocates its staging)
     st_b, out_b = _host_buffers(wl, r, n_inst)      # br_step_host_static (allocates nothing)
-    for k in range(2):                              # two calls in a row on the shared array
+    free_seen = []
+    for k in range(3):                              # calls in a row on the shared array
         probs = np.ascontiguousarray(wlm.term_probs_np(wl, k)) if cfg.H > 0 else None
         up_a, down_a = r.step_host(st_a, out_a, probs)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         up_b, down_b = r.step_host_static(st_b, out_b, probs)
+        torch.cuda.synchronize()
+        free_seen.append((free_before, torch.cuda.mem_get_info()[0]))
         assert (up_a, down_a) == (up_b, down_b)
         for key in out_a:                           # integer work: the tolerance is equality
             assert np.array_equal(out_a[key], out_b[key]), (name, k, key)
@@ -38,6 +44,10 @@ def test_static_staging_matches_allocating_entry_point(name, n_inst):
             assert np.array_equal(st_a[key], st_b[key]), (name, k, key)
         assert int(st_b["step"][0]) == k + 1
         assert (out_b["assign"][0] >= -1).all() and (out_b["trace"][0][:, 0] >= out_b["trace"][0][:, 1]).all()
+    # no device memory was taken: free memory is the same before and after the second and third call
+    # (the first call may load the library's kernels, which the driver places in device memory)
+    for before, after in free_seen[1:]:
+        assert after == before
     r.close()
 
 
