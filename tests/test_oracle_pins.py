@@ -739,3 +739,97 @@ def test_empirical_survival_estimator_is_the_truncated_expectation():
     # one recorded length v: inside the window the request surely ends after v - a more steps
     assert oracle.survival([50] * 7, 8, 45) == (5.0, 1.0, 5.0)
     assert oracle.survival([50] * 7, 8, 41)[0] == 8.0 and oracle.survival([50] * 7, 8, 50)[0] == 8.0
+
+
+# ---------------------------------------------------------------- lifetimes and perfect lookahead
+def test_requests_with_lifetimes_run_for_exactly_their_output_length():
+    """term_mode 3 (Section 2.2): a request admitted at step x with output length o runs at steps
+    x .. x + o - 1, its load growing by one token per step from s_i, and is gone at step x + o."""
+    G, B, W = 2, 3, 8
+    o = oracle.Instance(G=G, H=0, B=B, W=W, term_mode=3, S_greedy=0)
+    base = np.full((G, B), EMPTY, dtype=np.int32)
+    base[0, 0] = 40; base[1, 0] = 70                      # two running requests ...
+    qs = np.array([11, 22, 33, 0, 0, 0, 0, 0], np.int32)  # ... three waiting ones
+    o.set_state(0, 0, base, None, None, None, qs, None, 3)
+    end = np.zeros((G, B), np.int32); end[0, 0] = 2; end[1, 0] = 0      # last steps of the running ones
+    o.set_lifetimes(end, np.array([1, 3, 5, 0, 0, 0, 0, 0], np.int32))
+    seen = {}                                             # (worker, slot) -> loads step by step
+    for k in range(8):
+        st0 = o.get_state()
+        assign, load, _, _ = o.step()
+        st1 = o.get_state()
+        occ_after_admit = (st1["act_base"] != EMPTY)
+        # loads recorded at step k include everything that ran at step k
+        running = {}
+        for g in range(G):
+            for b in range(B):
+                was = st0["act_base"][g, b] != EMPTY
+                adm = bool((assign == g * B + b).any())
+                if was or adm:
+                    running[(g, b)] = True
+        for key in running:
+            seen.setdefault(key, []).append(k)
+    # the two initial requests: last steps 2 and 0
+    assert seen[(0, 0)] == [0, 1, 2] and seen[(1, 0)] == [0]
+    # admissions at step 0 (Stage 1 fills the emptiest worker first; both have two free slots, worker 0
+    # is lighter): whatever the placement, each admitted request runs for exactly o steps
+    lifetimes = sorted(len(v) for key, v in seen.items() if key not in ((0, 0), (1, 0)))
+    assert lifetimes == [1, 3, 5]
+
+
+def test_lifetime_loads_grow_by_one_token_per_step():
+    G, B = 1, 2
+    o = oracle.Instance(G=G, H=0, B=B, W=4, term_mode=3)
+    base = np.full((G, B), EMPTY, dtype=np.int32); base[0, 0] = 100
+    o.set_state(0, 0, base, None, None, None, np.array([7, 0, 0, 0], np.int32), None, 1)
+    o.set_lifetimes(np.array([[3, 0]], np.int32), np.array([2, 0, 0, 0], np.int32))
+    loads = [int(o.step()[1][0]) for _ in range(6)]
+    # step 0: 100 + 7; step 1: 101 + 8 (the admitted request's second and last step); step 2: 102;
+    # step 3: 103 (last step of the first request); then nothing runs
+    assert loads == [107, 109, 102, 103, 0, 0]
+
+
+def test_perfect_lookahead_is_min_of_remaining_steps_and_h():
+    """pred_mode 1 (Section 5.1 "Our methods", BR-H oracle): c_hat = min(r_i(k), H); with the offset
+    convention of the projection a request is counted at offsets h <= c_hat."""
+    G, B, H, k = 2, 4, 5, 10
+    o = oracle.Instance(G=G, H=H, B=B, W=4, term_mode=3, pred_mode=1, beta=4.0, gamma=0.5)
+    base = np.full((G, B), EMPTY, dtype=np.int32)
+    base[0, :3] = [100 - k, 200 - k, 300 - k]            # loads 100, 200, 300 at step k
+    base[1, :2] = [50 - k, 60 - k]
+    o.set_state(k, 0, base, None, None, None, None, None, 0)
+    end = np.zeros((G, B), np.int32)
+    end[0, :3] = [k, k + 2, k + 40]                       # r = 1, 3, 41
+    end[1, :2] = [k + 4, k + 5]                           # r = 5, 6
+    o.set_lifetimes(end, np.zeros(4, np.int32))
+    o.predict_only(None)
+    st = o.get_state()
+    assert st["chat"][0, :3].tolist() == [1.0, 3.0, 5.0] and st["chat"][1, :2].tolist() == [5.0, 5.0]
+    Lh, Mh, m = o.projection()
+    want0 = [100 + 200 + 300, 101 + 201 + 301, 202 + 302, 203 + 303, 304, 305]
+    want1 = [110 + h * 2 for h in range(6)]
+    assert Lh[0].tolist() == want0 and Lh[1].tolist() == want1
+    assert Mh.tolist() == [max(a, b) for a, b in zip(want0, want1)]
+
+
+def test_arrivals_carry_output_lengths_from_the_table():
+    """term_mode 3: arrival j of step k gets out_tab[word j % 4 of Philox block (k, j / 4, 3, 0)]."""
+    cfg = wlm.get_config("h80", arrival=("const", 6.0), init_queue=0, init_active=64)
+    wl = wlm.make_workload(cfg, n_instances=1)
+    o = oracle.instance_from_workload(wl, 0)
+    o.set_lifetimes(np.full((cfg.G, cfg.B), 10 ** 6, np.int32), wl.state["wq_o"][0])   # nobody leaves: no admissions
+    key = [int(wl.seeds[0]) & 0xFFFFFFFF, int(wl.seeds[0]) >> 32]
+    for k in range(5):
+        n0 = o.get_state()["wq_n"]
+        o.step(None)
+        st = o.get_state()
+        _, qo = o.get_lifetimes()
+        u = _philox_py([k, 0, 0, 0], key)[0]
+        n = int((u >= wl.arr_rows_for(0)[0].astype(np.int64)).sum())
+        # the workers are full and stay full, so every arrival stays in the queue
+        assert st["wq_n"] == n0 + n
+        for j in range(n):
+            r_len = _philox_py([k, j // 4, 1, 0], key)[j % 4]
+            r_out = _philox_py([k, j // 4, 3, 0], key)[j % 4]
+            assert st["wq_s"][n0 + j] == wl.len_tab[r_len >> 16]
+            assert qo[n0 + j] == wl.out_tab[r_out >> 16]
