@@ -292,6 +292,19 @@ int br_survival_chat(br_ctx *ctx, void *stream, const int32_t *hist_sorted, cons
                      int32_t n_hist, const int32_t *age, int64_t count, float *c_hat, double *p_fin,
                      double *mu_rem);
 
+/*
+ * Range-checked build (libbr_dbg.so, compiled with -DBR_BOUNDS; the paper has no counterpart).  In
+ * that build every per-instance array of the step kernels -- shared memory and global rows -- is
+ * indexed through a span that knows its length: an index outside it is counted and redirected to a
+ * sink, so nothing outside the array is read or written and the kernel ends normally.
+ * br_debug_bounds_hits synchronises the device and returns the count since the library was loaded;
+ * br_debug_bounds_selftest indexes a span over the four device ints it is given three times out of
+ * range (into the sink) and returns how many hits that added (3).  Both return -1 in the normal
+ * build, BR_ECUDA if a CUDA call fails.
+ */
+int br_debug_bounds_hits(void);
+int br_debug_bounds_selftest(int32_t *four_ints);
+
 /* Frees the context, its staging buffers and graph.  NULL is accepted. */
 int br_destroy(br_ctx *ctx);
 

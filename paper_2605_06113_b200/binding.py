@@ -55,7 +55,7 @@ class BrLoadOut(C.Structure):
 
 
 EXPORTS = ["br_create", "br_step", "br_graph_capture", "br_graph_step", "br_step_host",
-           "br_step_host_static",
+           "br_step_host_static", "br_debug_bounds_hits", "br_debug_bounds_selftest",
            "br_fscore", "br_best_subset", "br_bypass_dispatch", "br_survival_chat", "br_destroy", "br_strerror", "br_version"]
 
 _lib = None
@@ -92,6 +92,8 @@ def lib():
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.br_survival_chat.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.br_debug_bounds_hits.argtypes = []
+        L.br_debug_bounds_selftest.argtypes = [C.c_void_p]
         L.br_destroy.argtypes = [C.c_void_p]
         L.br_strerror.restype = C.c_char_p
         L.br_strerror.argtypes = [C.c_int]
@@ -100,6 +102,15 @@ def lib():
                 getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
+
+
+def use_library(path: Optional[str] = None) -> None:
+    """Makes lib() load another build of the library (the range-checked libbr_dbg.so); None goes
+    back to libbr.so.  Contexts created earlier keep the library they were created with only as
+    long as the caller keeps using them through it: close them first."""
+    global _lib, LIB_PATH
+    _lib = None
+    LIB_PATH = os.path.join(_HERE, "libbr.so") if path is None else path
 
 
 def _ptr(t) -> Optional[int]:

@@ -9,6 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbr.so")
+LIB_DEBUG = os.path.join(HERE, "libbr_dbg.so")          # the same sources with range-checked indexing (-DBR_BOUNDS)
 SOURCES = ["br_api.cu"]
 
 NVCC_FLAGS = [
@@ -18,10 +19,10 @@ NVCC_FLAGS = [
 ]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     # every file of csrc/ is a dependency: the kernels live in headers included by br_api.cu
     deps = glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cuh"))
     deps.append(os.path.join(os.path.dirname(HERE), "include", "br.h"))
@@ -29,16 +30,29 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _compile(lib: str, extra, verbose: bool) -> None:
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = lib + f".tmp{os.getpid()}"
+    cmd = [nvcc] + NVCC_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + \
+          ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
+    subprocess.check_call(cmd)
+    os.replace(tmp, lib)
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-              ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
-        subprocess.check_call(cmd)
-        os.replace(tmp, LIB)
+        _compile(LIB, [], verbose)
     return LIB
+
+
+def build_debug(force: bool = False) -> str:
+    """The range-checked library: every index into a per-instance array is checked and counted."""
+    if force or _stale(LIB_DEBUG):
+        _compile(LIB_DEBUG, ["-DBR_BOUNDS"], False)
+    return LIB_DEBUG
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--debug" in sys.argv:
+        print(build_debug(force="--force" in sys.argv))

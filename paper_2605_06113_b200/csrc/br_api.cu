@@ -724,6 +724,49 @@ int br_survival_chat(br_ctx *ctx, void *stream, const int32_t *hist_sorted, cons
     return BR_OK;
 }
 
+#ifdef BR_BOUNDS
+namespace {
+// indexes a four-element span at -1, 4 and 7 (one read, two writes): all three land in the sink
+__global__ void bounds_selftest_kernel(int *four)
+{
+    const auto s = br::mk_span(four, 4);
+    const int v = s[-1];
+    s[4] = v + 1;
+    *br::vec_at<int4>(s, 4) = make_int4(1, 2, 3, 4);
+    s[3] = 7;                                             // in range: not counted
+}
+}  // namespace
+#endif
+
+int br_debug_bounds_hits(void)
+{
+#ifdef BR_BOUNDS
+    unsigned h = 0;
+    BR_CUDA(cudaDeviceSynchronize());
+    BR_CUDA(cudaMemcpyFromSymbol(&h, br::g_bounds_hits, sizeof(h)));
+    return (int)(h > 0x7FFFFFFFu ? 0x7FFFFFFFu : h);
+#else
+    return -1;
+#endif
+}
+
+int br_debug_bounds_selftest(int32_t *four_ints)
+{
+#ifdef BR_BOUNDS
+    if (!four_ints) return BR_EINVAL;
+    const int before = br_debug_bounds_hits();
+    if (before < 0) return before;
+    bounds_selftest_kernel<<<1, 1>>>(four_ints);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "bounds self-test launch");
+    const int after = br_debug_bounds_hits();
+    return after < 0 ? after : after - before;
+#else
+    (void)four_ints;
+    return -1;
+#endif
+}
+
 int br_destroy(br_ctx *ctx)
 {
     if (!ctx) return BR_OK;

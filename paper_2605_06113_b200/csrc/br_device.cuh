@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <type_traits>
 
 namespace br {
 
@@ -12,6 +13,55 @@ constexpr long long kNoKey = (long long)0x8000000000000000ull;
 constexpr int kNoIdx = 0x7FFFFFFF;
 
 enum : uint32_t { kStreamArrCount = 0, kStreamArrLen = 1, kStreamTerm = 2, kStreamArrOut = 3 };
+
+// ---- range-checked build -------------------------------------------------------------------
+// With -DBR_BOUNDS every per-instance array of the step kernels (shared memory and global rows) is
+// a Span that knows its length: an index outside it is counted in g_bounds_hits and redirected to
+// a sink, so nothing outside the array is touched and the kernel ends normally (no trap, no
+// assert).  The host reads the count with br_debug_bounds_hits().  In the normal build span_t<T>
+// is a plain pointer and the helpers below vanish.
+#ifdef BR_BOUNDS
+__device__ unsigned long long g_bounds_sink[8];
+__device__ unsigned g_bounds_hits;
+
+template <typename T>
+struct Span {
+    T *p;
+    long long n;
+    __device__ Span() : p(nullptr), n(0) {}
+    __device__ Span(T *p_, long long n_) : p(p_), n(p_ ? (n_ < 0 ? 0 : n_) : 0) {}
+    __device__ explicit operator bool() const { return p != nullptr; }
+    __device__ T &operator[](long long i) const
+    {
+        if (i < 0 || i >= n) { atomicAdd(&g_bounds_hits, 1u); return *reinterpret_cast<T *>(g_bounds_sink); }
+        return p[i];
+    }
+    __device__ Span operator+(long long off) const { return Span(p ? p + off : nullptr, n - off); }
+};
+template <typename T> using span_t = Span<T>;
+template <typename T> __device__ __forceinline__ Span<T> mk_span(T *p, long long n) { return Span<T>(p, n); }
+// pointer to a vector of V that covers elements [i, i + sizeof(V) / sizeof(T)) of s
+template <typename V, typename T>
+__device__ __forceinline__ V *vec_at(const Span<T> &s, long long i)
+{
+    const long long cnt = (long long)(sizeof(V) / sizeof(T));
+    if (i < 0 || i + cnt > s.n) {
+        atomicAdd(&g_bounds_hits, 1u);
+        return reinterpret_cast<V *>(g_bounds_sink);
+    }
+    return reinterpret_cast<V *>(const_cast<typename std::remove_const<T>::type *>(s.p) + i);
+}
+template <typename T> __device__ __forceinline__ T *raw_of(const Span<T> &s) { return s.p; }
+#else
+template <typename T> using span_t = T *;
+template <typename T> __device__ __forceinline__ T *mk_span(T *p, long long) { return p; }
+template <typename V, typename T>
+__device__ __forceinline__ V *vec_at(T *p, long long i)
+{
+    return reinterpret_cast<V *>(const_cast<typename std::remove_const<T>::type *>(p) + i);
+}
+template <typename T> __device__ __forceinline__ T *raw_of(T *p) { return p; }
+#endif
 
 // First statements of a step kernel: let the next kernel of the stream start becoming resident,
 // then wait until every earlier kernel of the stream has completed and flushed its writes

@@ -74,7 +74,8 @@ __device__ void mitm_build(const int *win, int ra, unsigned long long *keys, int
 
 // Phase 2 for one subset of the high entries (mask_hi, its sum and size): updates b with the
 // neighbours of the peak among the admissible classes of the sorted half.
-__device__ __forceinline__ void mitm_probe(const unsigned long long *keys, const int *cls_off, int ra, int lim,
+template <typename KEYS, typename OFFS>
+__device__ __forceinline__ void mitm_probe(const KEYS keys, const OFFS cls_off, int ra, int lim,
                                            int peak, unsigned mask_hi, int sum_hi, int pop_hi, MitmBest &b)
 {
     const int cmax = min(ra, lim - pop_hi);

@@ -34,17 +34,20 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
     stream_order_gate();
     if (row >= a.N) return;
     const int inst = a.first_instance + row;
-    int *q_key = reinterpret_cast<int *>(smem_all) + wib * (2 * NT4 * 128);          // [NT4 * 128] packed keys
-    unsigned *q_id = reinterpret_cast<unsigned *>(q_key + NT4 * 128);                 // [NT4 * 128] request ids
+    int *q_key_p = reinterpret_cast<int *>(smem_all) + wib * (2 * NT4 * 128);
+    const auto q_key = mk_span(q_key_p, NT4 * 128);                                   // [NT4 * 128] packed keys
+    const auto q_id = mk_span(reinterpret_cast<unsigned *>(q_key_p + NT4 * 128), NT4 * 128);   // [NT4 * 128] request ids
 
     const int G = a.G, B = a.B, W = a.W, WL = a.wl, A = G * B;
     const unsigned posmask = (1u << WL) - 1u;
     const unsigned lt = (1u << lane) - 1u;
 
-    int32_t *g_base = a.ws.act_base + (size_t)inst * A;
-    uint32_t *g_aid = a.ws.act_id ? a.ws.act_id + (size_t)inst * A : nullptr;
-    int32_t *g_qs = a.wq.s + (size_t)inst * W;
-    uint32_t *g_qid = a.wq.id + (size_t)inst * W;
+    const auto g_base = mk_span(a.ws.act_base + (size_t)inst * A, A);
+    const auto g_aid = mk_span(a.ws.act_id ? a.ws.act_id + (size_t)inst * A : nullptr, A);
+    const auto g_qs = mk_span(a.wq.s + (size_t)inst * W, W);
+    const auto g_qid = mk_span(a.wq.id + (size_t)inst * W, W);
+    const auto t_len = mk_span(a.len_tab, a.len_tab ? (1ll << (32 - a.len_shift)) : 0);
+    const auto t_term = mk_span(a.term_cdf, B);
 
     const unsigned long long seed = a.ws.seed[inst];
     const uint32_t key0 = (uint32_t)seed, key1 = (uint32_t)(seed >> 32);
@@ -72,27 +75,27 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
         const int p0 = (t * 32 + lane) * 4;
         int4 sv = make_int4(0, 0, 0, 0); uint4 iv = make_uint4(0u, 0u, 0u, 0u);
         if (p0 < W) {
-            sv = *reinterpret_cast<const int4 *>(g_qs + p0);
-            iv = *reinterpret_cast<const uint4 *>(g_qid + p0);
+            sv = *vec_at<const int4>(g_qs, p0);
+            iv = *vec_at<const uint4>(g_qid, p0);
         }
         int4 kk;
         kk.x = p0 + 0 < n_w ? (sv.x << WL) | (int)(posmask - (unsigned)(p0 + 0)) : kSmallBeyond;
         kk.y = p0 + 1 < n_w ? (sv.y << WL) | (int)(posmask - (unsigned)(p0 + 1)) : kSmallBeyond;
         kk.z = p0 + 2 < n_w ? (sv.z << WL) | (int)(posmask - (unsigned)(p0 + 2)) : kSmallBeyond;
         kk.w = p0 + 3 < n_w ? (sv.w << WL) | (int)(posmask - (unsigned)(p0 + 3)) : kSmallBeyond;
-        *reinterpret_cast<int4 *>(q_key + p0) = kk;
-        *reinterpret_cast<uint4 *>(q_id + p0) = iv;
+        *vec_at<int4>(q_key, p0) = kk;
+        *vec_at<uint4>(q_id, p0) = iv;
     }
     __syncwarp();
 
 #pragma unroll 1
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + inst;          // outputs use the rows of the state (first_instance = 0 when n_steps > 1)
-        int32_t *assign = a.assign_out + orow * W;
+        const auto assign = mk_span(a.assign_out + orow * W, W);
 #pragma unroll
         for (int t = 0; t < NT4; ++t) {
             const int p0 = (t * 32 + lane) * 4;
-            if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(-1, -1, -1, -1);
+            if (p0 < W) *vec_at<int4>(assign, p0) = make_int4(-1, -1, -1, -1);
         }
 
         // ================= ARRIVE (Section 2.2) =================
@@ -102,7 +105,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
         uint4 rb = make_uint4(0u, 0u, 0u, 0u);
         if (a.arr_cdf) {
             const int kp = a.arr_period == 1 ? 0 : k % a.arr_period;
-            const uint32_t *rowp = a.arr_cdf + ((size_t)inst * a.arr_inst_stride + (size_t)kp) * a.arr_len;
+            const auto rowp = mk_span(a.arr_cdf + ((size_t)inst * a.arr_inst_stride + (size_t)kp) * a.arr_len, a.arr_len);
             const uint32_t r0 = lane < a.arr_len ? rowp[lane] : 0xFFFFFFFFu;
             const uint32_t r1 = lane + 32 < a.arr_len ? rowp[lane + 32] : 0xFFFFFFFFu;
             rb = philox4x32_10((uint32_t)k, lane == 31 ? 0u : (uint32_t)lane,
@@ -114,7 +117,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
         // constant-hazard draws of this step for worker `lane` (used after routing)
         unsigned long long fin = 0ull;
         if (a.term_mode == 1 && lane < G)
-            draw_ending(a.term_cdf, B, 1, (uint32_t)k, (uint32_t)lane, key0, key1, &fin);
+            draw_ending(t_term, B, 1, (uint32_t)k, (uint32_t)lane, key0, key1, &fin);
         // a request that was running before this step and ends at it: its load is asked for now
         const unsigned long long pre = occ & fin & slots;
         const int pj = __ffsll((long long)pre) - 1;
@@ -134,7 +137,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
             const uint32_t w2 = __shfl_sync(kFull, rb.z, src), w3 = __shfl_sync(kFull, rb.w, src);
             if (j < n_take) {
                 const uint32_t w = (j & 2) ? ((j & 1) ? w3 : w2) : ((j & 1) ? w1 : w0);
-                const int s = a.len_tab[w >> a.len_shift];
+                const int s = t_len[w >> a.len_shift];
                 const int pos = n_w_old + j;
                 q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
                 q_id[pos] = id0 + (unsigned)j;
@@ -177,7 +180,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
                     for (int r = 0; r < RM; ++r) tk[r] = 0;
 #pragma unroll
                     for (int t = 0; t < NT4; ++t) {
-                        const int4 kk = *reinterpret_cast<const int4 *>(q_key + (t * 32 + lane) * 4);
+                        const int4 kk = *vec_at<const int4>(q_key, (t * 32 + lane) * 4);
                         const int ke[4] = {kk.x, kk.y, kk.z, kk.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -218,7 +221,7 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
                 int bf = kEmpty, bkey = 0;
 #pragma unroll
                 for (int t = 0; t < NT4; ++t) {
-                    const int4 kk = *reinterpret_cast<const int4 *>(q_key + (t * 32 + lane) * 4);
+                    const int4 kk = *vec_at<const int4>(q_key, (t * 32 + lane) * 4);
                     const int ke[4] = {kk.x, kk.y, kk.z, kk.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -271,14 +274,14 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
 
         // ================= RECORD (Section 3.1) =================
         {
-            long long *o_load = reinterpret_cast<long long *>(a.out.load) + orow * G;
+            const auto o_load = mk_span(reinterpret_cast<long long *>(a.out.load) + orow * G, G);
             if (lane < G) o_load[lane] = (long long)L;
             const int mn = (int)__reduce_min_sync(kFull, lane < G ? (unsigned)L : 0xFFFFFFFFu);
             const unsigned lo = __reduce_add_sync(kFull, (unsigned)L & 0xFFFFu);
             const unsigned hi = __reduce_add_sync(kFull, (unsigned)L >> 16);
             status = (int)__reduce_or_sync(kFull, (unsigned)status);
             if (lane == 0) {
-                long long *tr = reinterpret_cast<long long *>(a.out.trace) + orow * 3;
+                const auto tr = mk_span(reinterpret_cast<long long *>(a.out.trace) + orow * 3, 3);
                 tr[0] = (long long)M; tr[1] = (long long)mn;
                 tr[2] = ((long long)hi << 16) + (long long)lo;
                 if (a.out.counters) {
@@ -299,8 +302,8 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
                 const int p0 = (t * 32 + lane) * 4;
                 if (t * 128 >= n_w) break;
                 if (t * 128 + 128 <= first_rm) { run += 128; continue; }     // nothing before the first admission moves
-                const int4 kk = *reinterpret_cast<const int4 *>(q_key + p0);
-                const uint4 ii = *reinterpret_cast<const uint4 *>(q_id + p0);
+                const int4 kk = *vec_at<const int4>(q_key, p0);
+                const uint4 ii = *vec_at<const uint4>(q_id, p0);
                 const int ke[4] = {kk.x, kk.y, kk.z, kk.w};
                 const unsigned idv[4] = {ii.x, ii.y, ii.z, ii.w};
                 int below = run;
@@ -353,12 +356,12 @@ __global__ void __maxnreg__(NT4 <= 2 ? 72 : 128) br_small_kernel(const StepArgs 
     for (int t = 0; t < NT4; ++t) {
         const int p0 = (t * 32 + lane) * 4;
         if (p0 < W) {
-            const int4 kk = *reinterpret_cast<const int4 *>(q_key + p0);
+            const int4 kk = *vec_at<const int4>(q_key, p0);
             int4 sv;
             sv.x = kk.x > 0 ? kk.x >> WL : 0; sv.y = kk.y > 0 ? kk.y >> WL : 0;
             sv.z = kk.z > 0 ? kk.z >> WL : 0; sv.w = kk.w > 0 ? kk.w >> WL : 0;
-            *reinterpret_cast<int4 *>(g_qs + p0) = sv;
-            *reinterpret_cast<uint4 *>(g_qid + p0) = *reinterpret_cast<const uint4 *>(q_id + p0);
+            *vec_at<int4>(g_qs, p0) = sv;
+            *vec_at<uint4>(g_qid, p0) = *vec_at<const uint4>(q_id, p0);
         }
     }
     if (lane < G) {

@@ -81,7 +81,7 @@ template <bool FP, int HM, bool SL = false>
 struct Scorer {
     int mi;                 // Eq. 1 margin
     double md[SL ? 1 : HM + 1];   // Eq. 2 margins
-    const double *mds;      // Eq. 2 margins in shared memory (SL)
+    span_t<double> mds;     // Eq. 2 margins in shared memory (SL)
     int mmin;               // min_h m_{g,h}: at or below it the Eq. 2 penalty is exactly zero
 
     __device__ __forceinline__ long long key(const StepArgs &a, int delta) const
@@ -149,9 +149,10 @@ __device__ __forceinline__ int warp_argmax_lane32(int key, unsigned tie, int &wk
 // Slots end independently with one probability, so the ending ones are walked by their gaps:
 // cdf[j] = floor(2^32 P(gap <= j)), draw t is word t % 4 of the Philox block (k, g, TERM, t / 4),
 // and a word u skips gap = #{j : u >= cdf[j]} slots (cdf ascends: the first j with u < cdf[j]).
-__device__ __forceinline__ void draw_ending(const uint32_t *__restrict__ cdf, int B, int OW, uint32_t k,
+template <typename CDF, typename OUT>
+__device__ __forceinline__ void draw_ending(const CDF cdf, int B, int OW, uint32_t k,
                                             uint32_t g, uint32_t key0, uint32_t key1,
-                                            unsigned long long *out)
+                                            const OUT out)
 {
     for (int w = 0; w < OW; ++w) out[w] = 0ull;
     int pos = 0;
@@ -161,11 +162,11 @@ __device__ __forceinline__ void draw_ending(const uint32_t *__restrict__ cdf, in
         if (t != 0u && (t & 3u) == 0u) r = philox4x32_10(k, g, kStreamTerm, t >> 2, key0, key1);
         const uint32_t u = word_of(r, t & 3u);
         const int room = B - pos;
-        if (u >= __ldg(cdf + room - 1)) break;            // the gap reaches past the last slot
+        if (u >= cdf[room - 1]) break;                    // the gap reaches past the last slot
         int lo = 0, hi = room - 1;                        // u < cdf[hi]
         while (lo < hi) {
             const int mid = (lo + hi) >> 1;
-            if (u < __ldg(cdf + mid)) hi = mid; else lo = mid + 1;
+            if (u < cdf[mid]) hi = mid; else lo = mid + 1;
         }
         const int slot = pos + lo;
         out[slot >> 6] |= 1ull << (slot & 63);
@@ -196,7 +197,8 @@ __device__ __forceinline__ void ld_row8(const float *p, float *o)
 // Adds (val, 1) to the prediction bucket `key` (load sum in T, count in C) if key >= 0.  Plain
 // shared-memory atomics: combining the lanes of a warp that share a bucket first (match.any and a
 // masked reduction) measured 70 % slower than letting the atomics collide.
-__device__ __forceinline__ void bucket_add(unsigned *T, unsigned *C, int key, unsigned val, int lane)
+template <typename TP, typename CP>
+__device__ __forceinline__ void bucket_add(const TP T, const CP C, int key, unsigned val, int lane)
 {
     (void)lane;
     if (key >= 0) { atomicAdd(&T[key], val); atomicAdd(&C[key], 1u); }
@@ -242,45 +244,67 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     const unsigned t_entry = (unsigned)clock64();
 
     // ---- shared-memory carve-up (sizes match step_smem_bytes) ----
-    int *q_key = reinterpret_cast<int *>(smem_raw);                                 // [W]
-    unsigned *q_id = reinterpret_cast<unsigned *>(q_key + W);                       // [W]
-    unsigned long long *occ = reinterpret_cast<unsigned long long *>(q_id + W);     // [G][OW]
-    unsigned long long *end_mask = occ + (size_t)G * OW;                            // [G][OW]
-    unsigned long long *fin_w = end_mask + (size_t)G * OW;                          // [G][OW] slots whose draw says "ends"
-    double *md_s = reinterpret_cast<double *>(fin_w + (size_t)G * OW);              // [H1] margins of the selected worker
-    int *M_s = reinterpret_cast<int *>(md_s + H1);                                  // [H1 rounded up to even] envelope
-    unsigned *Lh_s = reinterpret_cast<unsigned *>(M_s + (H1 + 1) / 2 * 2);          // [G][H1]
-    unsigned *Ch_s = Lh_s + (size_t)G * H1;                                         // [G][H1]
-    unsigned *sub_load = Ch_s + (size_t)G * H1;                                     // [G]
-    unsigned short *end_list = reinterpret_cast<unsigned short *>(sub_load + G);    // [kEndList]
-    unsigned short *pre_list = end_list + kEndList;                                 // [32]
-    int *scal = reinterpret_cast<int *>(pre_list + 32);
-    unsigned short *refresh_list = reinterpret_cast<unsigned short *>(scal + 16);   // [A] (H > 0 only)
+    // (raw carve-up first; every array is then used through a span that knows its length)
+    int *q_key_p = reinterpret_cast<int *>(smem_raw);                               // [W]
+    unsigned *q_id_p = reinterpret_cast<unsigned *>(q_key_p + W);                   // [W]
+    unsigned long long *occ_p = reinterpret_cast<unsigned long long *>(q_id_p + W); // [G][OW]
+    unsigned long long *end_mask_p = occ_p + (size_t)G * OW;                        // [G][OW]
+    unsigned long long *fin_w_p = end_mask_p + (size_t)G * OW;                      // [G][OW] slots whose draw says "ends"
+    double *md_s_p = reinterpret_cast<double *>(fin_w_p + (size_t)G * OW);          // [H1] margins of the selected worker
+    int *M_s_p = reinterpret_cast<int *>(md_s_p + H1);                              // [H1 rounded up to even] envelope
+    unsigned *Lh_s_p = reinterpret_cast<unsigned *>(M_s_p + (H1 + 1) / 2 * 2);      // [G][H1]
+    unsigned *Ch_s_p = Lh_s_p + (size_t)G * H1;                                     // [G][H1]
+    unsigned *sub_load_p = Ch_s_p + (size_t)G * H1;                                 // [G]
+    unsigned short *end_list_p = reinterpret_cast<unsigned short *>(sub_load_p + G);// [kEndList]
+    unsigned short *pre_list_p = end_list_p + kEndList;                             // [32]
+    int *scal_p = reinterpret_cast<int *>(pre_list_p + 32);                         // [16]
+    unsigned short *refresh_list_p = reinterpret_cast<unsigned short *>(scal_p + 16);   // [A] (H > 0 only)
     // output lengths of the waiting requests (term_mode 3 only), behind everything else
-    int *q_o = reinterpret_cast<int *>(smem_raw + ((step_smem_bytes(G, H, B, W, OW) + 15) & ~(size_t)15));
+    int *q_o_p = reinterpret_cast<int *>(smem_raw + ((step_smem_bytes(G, H, B, W, OW) + 15) & ~(size_t)15));
     // large Stage-2 windows: sorted subsets of the low half, class offsets, the window's keys
-    unsigned long long *bw_keys = reinterpret_cast<unsigned long long *>(
+    unsigned long long *bw_keys_p = reinterpret_cast<unsigned long long *>(
         smem_raw + step_smem_bytes(G, H, B, W, OW, !LEAN && a.term_mode == 3));
-    int *bw_off = reinterpret_cast<int *>(bw_keys + (1 << kBigWinLow));
-    int *bw_win = bw_off + 16;
+    int *bw_off_p = reinterpret_cast<int *>(bw_keys_p + (1 << kBigWinLow));
+    const bool life = !LEAN && a.term_mode == 3;          // requests carry their output lengths
+    const bool bigw = !LEAN && a.big_window != 0;
+    const auto q_key = mk_span(q_key_p, W);
+    const auto q_id = mk_span(q_id_p, W);
+    const auto occ = mk_span(occ_p, G * OW);
+    const auto end_mask = mk_span(end_mask_p, G * OW);
+    const auto fin_w = mk_span(fin_w_p, G * OW);
+    const auto md_s = mk_span(md_s_p, H1);
+    const auto M_s = mk_span(M_s_p, H1);
+    const auto Lh_s = mk_span(Lh_s_p, 2 * G * H1);        // Ch_s follows it; the two are cleared as one block
+    const auto Ch_s = mk_span(Ch_s_p, G * H1);
+    const auto sub_load = mk_span(sub_load_p, G);
+    const auto end_list = mk_span(end_list_p, kEndList);
+    const auto pre_list = mk_span(pre_list_p, 32);
+    const auto scal = mk_span(scal_p, 16);
+    const auto refresh_list = mk_span(refresh_list_p, H > 0 ? A : 0);
+    const auto q_o = mk_span(q_o_p, life ? W : 0);
+    const auto bw_keys = mk_span(bw_keys_p, bigw ? (1 << kBigWinLow) : 0);
+    const auto bw_off = mk_span(bw_off_p, bigw ? 16 : 0);
+    const auto bw_win = mk_span(bw_off_p + 16, bigw ? 16 : 0);
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
     //       [6] requests that ended this step and were not prefetched, [7] prefetched ones,
     //       [8] requests whose c_hat is refreshed at this step
 
     // ---- per-instance global rows ----
-    long long *g_load = reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G;
-    int32_t *g_nact = a.ws.nact + (size_t)inst * G;
-    unsigned long long *g_occ = reinterpret_cast<unsigned long long *>(a.ws.occ) + (size_t)inst * G * OW;
-    int32_t *g_base = a.ws.act_base + (size_t)inst * A;
-    uint32_t *g_aid = a.ws.act_id ? a.ws.act_id + (size_t)inst * A : nullptr;
-    float *g_chat0 = a.ws.act_chat0 ? a.ws.act_chat0 + (size_t)inst * A : nullptr;
-    uint8_t *g_kref = a.ws.act_kref ? a.ws.act_kref + (size_t)inst * A : nullptr;
-    const bool life = !LEAN && a.term_mode == 3;          // requests carry their output lengths
-    int32_t *g_end = life ? a.ws.act_end + (size_t)inst * A : nullptr;
-    int32_t *g_qo = life ? a.wq.o + (size_t)inst * W : nullptr;
-    int32_t *g_qs = a.wq.s + (size_t)inst * W;
-    uint32_t *g_qid = a.wq.id + (size_t)inst * W;
+    const auto g_load = mk_span(reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G, G);
+    const auto g_nact = mk_span(a.ws.nact + (size_t)inst * G, G);
+    const auto g_occ = mk_span(reinterpret_cast<unsigned long long *>(a.ws.occ) + (size_t)inst * G * OW, G * OW);
+    const auto g_base = mk_span(a.ws.act_base + (size_t)inst * A, A);
+    const auto g_aid = mk_span(a.ws.act_id ? a.ws.act_id + (size_t)inst * A : nullptr, A);
+    const auto g_chat0 = mk_span(a.ws.act_chat0 ? a.ws.act_chat0 + (size_t)inst * A : nullptr, A);
+    const auto g_kref = mk_span(a.ws.act_kref ? a.ws.act_kref + (size_t)inst * A : nullptr, A);
+    const auto g_end = mk_span(life ? a.ws.act_end + (size_t)inst * A : nullptr, A);
+    const auto g_qo = mk_span(life ? a.wq.o + (size_t)inst * W : nullptr, W);
+    const auto g_qs = mk_span(a.wq.s + (size_t)inst * W, W);
+    const auto g_qid = mk_span(a.wq.id + (size_t)inst * W, W);
+    const auto t_len = mk_span(a.len_tab, a.len_tab ? (1ll << (32 - a.len_shift)) : 0);
+    const auto t_out = mk_span(a.out_tab, a.out_tab ? (1ll << (32 - a.out_shift)) : 0);
+    const auto t_term = mk_span(a.term_cdf, B);
 
     const unsigned long long seed = a.ws.seed[inst];
     const uint32_t key0 = (uint32_t)seed, key1 = (uint32_t)(seed >> 32);
@@ -294,16 +318,16 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     // queue -> packed keys and ids in shared memory (16-byte loads).  The first chunks are
     // requested without waiting for the queue length (rows always hold W entries).
     auto fetch_queue = [&](int i) {
-        const int4 v = *reinterpret_cast<const int4 *>(g_qs + i);
-        const uint4 u = *reinterpret_cast<const uint4 *>(g_qid + i);
+        const int4 v = *vec_at<const int4>(g_qs, i);
+        const uint4 u = *vec_at<const uint4>(g_qid, i);
         int4 kk;
         kk.x = (v.x << WL) | (int)(posmask - (unsigned)(i + 0));
         kk.y = (v.y << WL) | (int)(posmask - (unsigned)(i + 1));
         kk.z = (v.z << WL) | (int)(posmask - (unsigned)(i + 2));
         kk.w = (v.w << WL) | (int)(posmask - (unsigned)(i + 3));
-        *reinterpret_cast<int4 *>(q_key + i) = kk;
-        *reinterpret_cast<uint4 *>(q_id + i) = u;
-        if (life) *reinterpret_cast<int4 *>(q_o + i) = *reinterpret_cast<const int4 *>(g_qo + i);
+        *vec_at<int4>(q_key, i) = kk;
+        *vec_at<uint4>(q_id, i) = u;
+        if (life) *vec_at<int4>(q_o, i) = *vec_at<const int4>(g_qo, i);
     };
     {
         const int i0 = tid * 4, i1 = (NT + tid) * 4;
@@ -319,7 +343,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     int cap[GW];
     int L[GW][HR + 1];
     int Mh[HR + 1];
-    int *const L_s = reinterpret_cast<int *>(Lh_s);     // SL: the buckets become L_g(k+h) in place
+    const auto L_s = mk_span(reinterpret_cast<int *>(raw_of(Lh_s)), G * H1);     // SL: the buckets become L_g(k+h) in place
 #pragma unroll
     for (int h = 0; h <= HR; ++h) Mh[h] = 0;
 #pragma unroll
@@ -342,7 +366,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     auto draw_fin = [&](int first, int stride) {
 #pragma unroll 1
         for (int g = first; g < G; g += stride)
-            draw_ending(a.term_cdf, B, OW, (uint32_t)k, (uint32_t)g, key0, key1, fin_w + (size_t)g * OW);
+            draw_ending(t_term, B, OW, (uint32_t)k, (uint32_t)g, key0, key1, fin_w + (size_t)g * OW);
     };
 
     // Per worker word: which running requests end at this step (occupancy & termination draws).
@@ -378,7 +402,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
 
     for (int it = 0; it < a.n_steps; ++it, ++k) {
         const size_t orow = (size_t)it * a.N + inst;
-        const float *probs = a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr;
+        const auto probs = mk_span(a.term_probs ? a.term_probs + orow * (size_t)A * H : nullptr, (long long)A * H);
         unsigned t_phase[7];
         const bool timing = !LEAN && a.out.phase_cycles != nullptr && tid == 0;
         if (timing) t_phase[0] = (unsigned)clock64();
@@ -387,9 +411,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // the arrival-count row is requested first; a single-warp block draws the termination
         // words while that load is in flight
         uint32_t row0 = 0xFFFFFFFFu, row1 = 0xFFFFFFFFu;
-        const uint32_t *row = nullptr;
+        span_t<const uint32_t> row = mk_span((const uint32_t *)nullptr, 0);
         if (a.arr_cdf) {
-            row = a.arr_cdf + ((size_t)inst * a.arr_inst_stride + (size_t)(k % a.arr_period)) * a.arr_len;
+            row = mk_span(a.arr_cdf + ((size_t)inst * a.arr_inst_stride + (size_t)(k % a.arr_period)) * a.arr_len, a.arr_len);
             if (lane < a.arr_len) row0 = row[lane];
             if (lane + 32 < a.arr_len) row1 = row[lane + 32];
         }
@@ -424,12 +448,12 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             const int pos = n_w_old + j;
             if (pos < W) {
                 const uint4 r = philox4x32_10((uint32_t)k, (uint32_t)j >> 2, kStreamArrLen, 0u, key0, key1);
-                const int s = a.len_tab[word_of(r, j & 3) >> a.len_shift];
+                const int s = t_len[word_of(r, j & 3) >> a.len_shift];
                 q_key[pos] = (s << WL) | (int)(posmask - (unsigned)pos);
                 q_id[pos] = id0 + (unsigned)j;
                 if (life) {
                     const uint4 ro = philox4x32_10((uint32_t)k, (uint32_t)j >> 2, kStreamArrOut, 0u, key0, key1);
-                    q_o[pos] = a.out_tab[word_of(ro, j & 3) >> a.out_shift];
+                    q_o[pos] = t_out[word_of(ro, j & 3) >> a.out_shift];
                 }
             }
         }
@@ -451,8 +475,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             for (int q0 = 0; q0 < A4; q0 += NT) {
                 const int q4 = q0 + tid;
                 const bool inr = q4 < A4;
-                const int4 bq = inr ? *reinterpret_cast<const int4 *>(g_base + 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
-                const int4 eq = inr ? *reinterpret_cast<const int4 *>(g_end + 4 * q4) : make_int4(0, 0, 0, 0);
+                const int4 bq = inr ? *vec_at<const int4>(g_base, 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
+                const int4 eq = inr ? *vec_at<const int4>(g_end, 4 * q4) : make_int4(0, 0, 0, 0);
                 const int bs4[4] = {bq.x, bq.y, bq.z, bq.w};
                 const int en4[4] = {eq.x, eq.y, eq.z, eq.w};
                 const int g = (int)__umulhi((unsigned)(4 * q4), a.magic_B);
@@ -473,9 +497,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 for (int u = 0; u < kUnroll; ++u) {
                     const int q4 = q_base + u * NT + tid;
                     const bool inr = q4 < A4;
-                    bq[u] = inr ? *reinterpret_cast<const int4 *>(g_base + 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
-                    cq[u] = inr ? *reinterpret_cast<const float4 *>(g_chat0 + 4 * q4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    kq[u] = inr ? *reinterpret_cast<const unsigned *>(g_kref + 4 * q4) : 0u;
+                    bq[u] = inr ? *vec_at<const int4>(g_base, 4 * q4) : make_int4(kEmpty, kEmpty, kEmpty, kEmpty);
+                    cq[u] = inr ? *vec_at<const float4>(g_chat0, 4 * q4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    kq[u] = inr ? *vec_at<const unsigned>(g_kref, 4 * q4) : 0u;
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
@@ -525,7 +549,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 unsigned cur = 0u;
                 if (e < n_ref) {
                     const int s0 = refresh_list[e];
-                    const float *q = probs + (size_t)s0 * H;
+                    const auto q = probs + (long long)s0 * H;
                     double v = (double)H;                               // gate closed: the conservative anchor
                     if (SL) {
                         // long classifier rows stay in memory: p_fin and c* in one pass
@@ -537,13 +561,13 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         if (__dsub_rn(1.0, surv) >= (double)a.gate) v = cs;
                     } else {
                         float qv[HR > 0 ? HR : 1];
-                        if (HR == 8 && H == 8 && (reinterpret_cast<size_t>(probs) & 31) == 0) {
-                            ld_row8(q, qv);
+                        if (HR == 8 && H == 8 && (reinterpret_cast<size_t>(raw_of(probs)) & 31) == 0) {
+                            ld_row8(reinterpret_cast<const float *>(vec_at<const double4>(q, 0)), qv);
                         } else if ((H & 3) == 0) {
 #pragma unroll
                             for (int h = 0; h < HR; h += 4) {
                                 if (h < H) {
-                                    const float4 qq = ld_row4(q + h);
+                                    const float4 qq = ld_row4(reinterpret_cast<const float *>(vec_at<const float4>(q, h)));
                                     qv[h] = qq.x; qv[h + 1] = qq.y; qv[h + 2] = qq.z; qv[h + 3] = qq.w;
                                 }
                             }
@@ -1112,7 +1136,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
             {
                 int mx = L[0][0], mn = cap[0] >= 0 ? L[0][0] : 0x7FFFFFFF;
                 long long sum = cap[0] >= 0 ? (long long)L[0][0] : 0;
-                long long *o_load = reinterpret_cast<long long *>(a.out.load) + orow * G;
+                const auto o_load = mk_span(reinterpret_cast<long long *>(a.out.load) + orow * G, G);
                 if (cap[0] >= 0) o_load[lane] = L[0][0];
 #pragma unroll
                 for (int w = 1; w < GW; ++w) {
@@ -1126,7 +1150,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
                 status = (int)__reduce_or_sync(kFull, (unsigned)status);
                 if (lane == 0) {
-                    long long *tr = reinterpret_cast<long long *>(a.out.trace) + orow * 3;
+                    const auto tr = mk_span(reinterpret_cast<long long *>(a.out.trace) + orow * 3, 3);
                     tr[0] = mx; tr[1] = mn; tr[2] = sum;
                     scal[0] = n_left; scal[1] = admitted; scal[2] = s1_iters; scal[3] = s2_pops;
                     scal[4] = status | (n_drop ? BR_ST_QUEUE_OVERFLOW : 0);
@@ -1142,7 +1166,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
         // A lane owns four consecutive positions of every group of 128 (16-byte accesses to the keys,
         // the ids and the assignment row); an entry's new position is the count of kept entries before it.
         if (warp == 0) {
-            int32_t *assign = a.assign_out + orow * W;
+            const auto assign = mk_span(a.assign_out + orow * W, W);
             int run = 0;
             const int n_before = n_w;          // queue length after ARRIVE
             const unsigned lt = (1u << lane) - 1u;
@@ -1151,14 +1175,14 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 const int p0 = i0 + lane * 4;
                 if (i0 >= n_before) {
                     // the rest of the row is beyond the queue: only assignments remain
-                    if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(-1, -1, -1, -1);
+                    if (p0 < W) *vec_at<int4>(assign, p0) = make_int4(-1, -1, -1, -1);
                     continue;
                 }
                 int4 kk = make_int4(0, 0, 0, 0); uint4 ii = make_uint4(0u, 0u, 0u, 0u); int4 oo = make_int4(0, 0, 0, 0);
                 if (p0 < W) {
-                    kk = *reinterpret_cast<const int4 *>(q_key + p0);
-                    ii = *reinterpret_cast<const uint4 *>(q_id + p0);
-                    if (life) oo = *reinterpret_cast<const int4 *>(q_o + p0);
+                    kk = *vec_at<const int4>(q_key, p0);
+                    ii = *vec_at<const uint4>(q_id, p0);
+                    if (life) oo = *vec_at<const int4>(q_o, p0);
                 }
                 int ke[4] = {kk.x, kk.y, kk.z, kk.w};
                 const unsigned idv[4] = {ii.x, ii.y, ii.z, ii.w};
@@ -1189,7 +1213,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         }
                     }
                 }
-                if (p0 < W) *reinterpret_cast<int4 *>(assign + p0) = make_int4(as[0], as[1], as[2], as[3]);
+                if (p0 < W) *vec_at<int4>(assign, p0) = make_int4(as[0], as[1], as[2], as[3]);
                 __syncwarp();                                           // the group is read before any of it is overwritten
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -1238,7 +1262,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                             }
                         }
                     }
-                    reinterpret_cast<unsigned char *>(fin_w + (size_t)g * OW)[slot0 >> 3] = (unsigned char)fb;
+                    *vec_at<unsigned char>(mk_span(reinterpret_cast<unsigned char *>(raw_of(fin_w)), (long long)G * OW * 8), (long long)g * OW * 8 + (slot0 >> 3)) = (unsigned char)fb;
                 }
                 inst_sync();
             } else if (term_mode == 3) {
@@ -1250,13 +1274,13 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     const unsigned ob = (unsigned)(occ[g * OW + (slot0 >> 6)] >> (slot0 & 63)) & 0xFFu;
                     unsigned fb = 0;
                     if (ob) {
-                        const int4 e0 = *reinterpret_cast<const int4 *>(g_end + a0);
-                        const int4 e1 = *reinterpret_cast<const int4 *>(g_end + a0 + 4);
+                        const int4 e0 = *vec_at<const int4>(g_end, a0);
+                        const int4 e1 = *vec_at<const int4>(g_end, a0 + 4);
                         const int en[8] = {e0.x, e0.y, e0.z, e0.w, e1.x, e1.y, e1.z, e1.w};
 #pragma unroll
                         for (int j = 0; j < 8; ++j) if (((ob >> j) & 1u) && en[j] == k) fb |= 1u << j;
                     }
-                    reinterpret_cast<unsigned char *>(fin_w + (size_t)g * OW)[slot0 >> 3] = (unsigned char)fb;
+                    *vec_at<unsigned char>(mk_span(reinterpret_cast<unsigned char *>(raw_of(fin_w)), (long long)G * OW * 8), (long long)g * OW * 8 + (slot0 >> 3)) = (unsigned char)fb;
                 }
                 inst_sync();
             }
