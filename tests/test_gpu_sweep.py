@@ -61,9 +61,8 @@ def test_beta_gamma_cross_at_h80():
     lines += [f"| {n} | {v:,.0f} | {v / rr:.2f} |" for n, v in rows]
     text = "\n".join(lines)
     print("\n" + text)
-    out_dir = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(out_dir):
-        with open(os.path.join(out_dir, "sweep_h80.md"), "w") as f:
+    if os.environ.get("BR_SWEEP_TABLE"):                       # optional copy of the table as a file
+        with open(os.environ["BR_SWEEP_TABLE"], "w") as f:
             f.write(text + "\n")
     centre = dict(rows)["BR-H (beta = 48, gamma = 0.9)"]
     # the paper's qualitative finding on its traces: BR-H below BR-0 below the load-blind router,
