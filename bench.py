@@ -205,7 +205,7 @@ def _oracle_worker(job):
     cfg = wlm.get_config(cfg_name)
     wl = wlm.make_workload(cfg, n_instances=n, first_instance=first)
     orcs = [oracle.instance_from_workload(wl, i) for i in range(n)]
-    probs = [wlm.term_probs_np(wl, k) for k in range(min(max_steps, 4))] if cfg.H > 0 else None
+    probs = [wlm.term_probs_np(wl, k) for k in range(min(max_steps, 4))] if cfg.H > 0 and cfg.pred_mode == 0 else None
     done = 0
     t0 = time.perf_counter()
     for k in range(max_steps):
@@ -319,7 +319,7 @@ class RotatingSets:
             st0 = {k: v.clone() for k, v in st.items()}
             out = router.outputs(n_inst, n_steps=spl)
             probs = []
-            if self.cfg.H > 0:
+            if self.cfg.H > 0 and self.cfg.pred_mode == 0:      # classifier rows (the perfect-lookahead predictor reads none)
                 seeds_t = torch.from_numpy(wl.seeds.astype(np.int64)).to(device)
                 tab_t = torch.from_numpy(wl.beta_tab).to(device)
                 for j in range(max(1, probs_ring)):
@@ -389,7 +389,7 @@ def time_region(torch, fn, steps, dist=None):
 
 
 def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, threads=0,
-                    seed_offset=0, dist=None, sampler=None, probs_ring=2):
+                    seed_offset=0, dist=None, sampler=None, probs_ring=2, n_inst=None):
     """Times `launches` br_step calls of the batched configuration `wname`, `spl` decode steps per
     call, `repeats` times.  Enough instance sets rotate that the data between two visits of a set
     exceeds L2 and that no instance runs past the configuration's length.  The work of a decode
@@ -400,7 +400,7 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     repeat the sets return to their starting snapshots and one untimed call per set runs;
     `warmup` untimed calls precede the first repeat."""
     cfg = wlm.get_config(wname)
-    N = cfg.N
+    N = cfg.N if n_inst is None else n_inst
     per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
     n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
     n_sets = max(n_sets, int(np.ceil((launches + n_sets) * spl / cfg.steps)))
@@ -539,6 +539,16 @@ def run_ours(args):
         line["single_step_launches"] = {"value": m1["value"], "unit": UNIT, "ms_per_step": m1["ms_per_launch"],
                                         "roofline": r1, "gpu_launches": m1["launches"], "repeats_ms": m1["repeats_ms"]}
         summary["c3_1_step_per_launch"] = brief(m1, r1)
+        # two batches in one call (8,192 instances, one decode step): the second wave of thread blocks
+        # fills the SMs that the first wave's short instances leave early
+        m2 = measure_batched(torch, wname, device, 200, 20, 1, repeats=5, threads=args.threads, n_inst=2 * N)
+        line["single_step_launches_8192_instances"] = {
+            "value": m2["value"], "unit": UNIT, "ms_per_step": m2["ms_per_launch"], "instances_per_launch": 2 * N,
+            "us_per_4096_instance_steps": m2["us_per_launch"] / 2, "repeats_ms": m2["repeats_ms"],
+            "frac": m2["achieved"] / peak}
+        summary["c3_1_step_per_launch_8192_instances"] = {
+            "us_per_launch": round(m2["us_per_launch"], 2), "us_per_4096_instance_steps": round(m2["us_per_launch"] / 2, 2),
+            "inst_steps_per_s": round(m2["value"]), "frac": round(m2["achieved"] / peak, 4)}
         # ---------------- end to end through the host-buffer entry point ----------------
         line["e2e"] = e2e_host(torch, device, args)
         summary["e2e_c3_host_buffers"] = {"inst_steps_per_s": round(line["e2e"]["value"]),
@@ -602,6 +612,15 @@ def extras(torch, device, args, peak, peak_kind, summary):
         ex[key] = {"value": m["value"], "unit": UNIT, "ms_per_step": m["ms_per_launch"], "steps_per_launch": spl,
                    "repeats_ms": m["repeats_ms"], "roofline": roof}
         summary[f"c4_{spl}_step{'s' if spl > 1 else ''}_per_launch"] = brief(m, roof)
+    # the deployed lookahead as a batch: 1,024 instances of the h80 workload (H = 80, G = 8, R_max = 4), 8 steps per launch
+    try:
+        mh = measure_batched(torch, "h80", device, 24, 4, 8, repeats=5, n_inst=1024)
+        ex["h80_batched"] = {"value": mh["value"], "unit": UNIT, "ms_per_step": mh["ms_per_launch"], "steps_per_launch": 8,
+                             "instances_per_launch": 1024, "repeats_ms": mh["repeats_ms"]}
+        summary["h80_batched_1024_instances"] = {"us_per_decode_step": round(mh["us_per_launch"] / 8, 2),
+                                                 "inst_steps_per_s": round(mh["value"])}
+    except Exception as e:
+        ex["h80_batched"] = {"error": repr(e)}
     # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
     try:
         ex["entry_points"] = entry_points(torch, device, peak)
