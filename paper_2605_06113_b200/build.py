@@ -45,6 +45,22 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_all(force: bool = False) -> None:
+    """Both libraries, compiled side by side when both are out of date."""
+    import threading
+    jobs = []
+    if force or _stale():
+        jobs.append(threading.Thread(target=_compile, args=(LIB, [], False)))
+    if force or _stale(LIB_DEBUG):
+        jobs.append(threading.Thread(target=_compile, args=(LIB_DEBUG, ["-DBR_BOUNDS"], False)))
+    for j in jobs:
+        j.start()
+    for j in jobs:
+        j.join()
+    if not (os.path.exists(LIB) and os.path.exists(LIB_DEBUG)):
+        raise RuntimeError("building the CUDA libraries failed (see the compiler output above)")
+
+
 def build_debug(force: bool = False) -> str:
     """The range-checked library: every index into a per-instance array is checked and counted."""
     if force or _stale(LIB_DEBUG):
