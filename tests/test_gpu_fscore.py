@@ -12,9 +12,9 @@ from paper_2605_06113_b200.binding import Router
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,H", [("c3", 0), ("c4", 8), ("c2", 4)])
+@pytest.mark.parametrize("name,H", [("c3", 0), ("c4", 8), ("c2", 4), ("h80", 80), ("c4", 33)])
 def test_fscore_matrix_and_best_worker(name, H):
-    cfg = wlm.get_config(name)
+    cfg = wlm.get_config(name, H=H)
     wl = wlm.make_workload(cfg, n_instances=2)
     r = Router(wl, device="cuda:0")
     rng = np.random.default_rng(3 + H)

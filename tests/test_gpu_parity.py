@@ -282,3 +282,13 @@ def test_large_stage2_windows_random_shapes():
                              arrival=("const", float(rng.choice([2.0, 12.0]))), first_seed=3100 * case)
         run_parity(cfg, 2, 30, threads=int(rng.choice([0, 32, 128])), check_every=10,
                    launch_steps=int(rng.choice([1, 4])))
+
+
+def test_long_horizon_large_fleet_needs_more_than_48k_of_shared_memory():
+    """H = 80 on G = 64 workers with 1,024 waiting requests: about 60 KB of shared memory per instance,
+    beyond the default limit, so the kernel is opted in at launch."""
+    run_parity(wlm.get_config("c4", H=80, term_mode=1, gate=0.3, beta=48.0, gamma=0.9), 2, 12, check_every=4)
+    run_parity(wlm.get_config("h80", G=64, W=1024, init_queue=1000, arrival=("const", 5.0)), 2, 12, check_every=4,
+               threads=256)
+    run_parity(wlm.get_config("h80", G=64, W=1024, init_queue=1000, arrival=("const", 5.0)), 1, 8, check_every=4,
+               graph=True)                             # the opt-in also happens while a graph is captured
