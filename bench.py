@@ -6,9 +6,10 @@
 A "step" is one call of br_step: one launch of the whole routing path (ARRIVE, PREDICT, ROUTE,
 RECORD, ADVANCE) over one batch of 4,096 independent BR-0 instances (G = 32, 256 waiting each:
 the batched HBM-throughput configuration), advancing every instance by --steps-per-launch
-decode steps (16 unless asked otherwise; `config.steps_per_launch` says which).  The timed
+decode steps (16, or with a short timed region the number with which its calls cover the
+configuration once; `config.steps_per_launch` says which).  The timed
 region of --steps calls is repeated --repeats times, each repeat on instance sets put back to
-their starting snapshots and primed by untimed calls; the median repeat is reported, minimum and
+their starting snapshots; the median repeat is reported, minimum and
 maximum beside it.  Several instance sets are stepped in rotation so that the data touched
 between two visits of the same set exceeds the L2 cache; they start at evenly spaced points of
 the configuration's trajectory, so that a short timed region still samples all of it.  Prints one JSON line whose last key,
@@ -68,11 +69,22 @@ def kernel_source_hash() -> str:
 
 
 def _recorded(field: str, workload: str, spl: int):
+    """A per-launch counter from the ncu captures in profiles/traffic.json.  For a launch shape that
+    was not captured itself the figure is interpolated linearly in the steps per launch between
+    the two shapes that were (the first step of a launch reads the state from DRAM, every further
+    step adds the same amount)."""
     p = os.path.join(ROOT, "profiles", "traffic.json")
     try:
         rec = json.load(open(p))
-        if rec.get("kernel_source_hash") == kernel_source_hash():
-            return rec.get(field, {}).get(f"{workload}_spl{spl}")
+        if rec.get("kernel_source_hash") != kernel_source_hash():
+            return None
+        tab = rec.get(field, {})
+        if f"{workload}_spl{spl}" in tab:
+            return tab[f"{workload}_spl{spl}"]
+        pts = sorted((int(k.rsplit("spl", 1)[1]), v) for k, v in tab.items() if k.startswith(workload + "_spl"))
+        if len(pts) >= 2:
+            (s0, v0), (s1, v1) = pts[0], pts[-1]
+            return v0 + (v1 - v0) * (spl - s0) / (s1 - s0)
     except Exception:
         pass
     return None
@@ -190,9 +202,16 @@ def dist_setup(args):
     return world, rank, local, None
 
 
-def steps_per_launch_for(cfg, asked: int) -> int:
-    """Decode steps per br_step call: what was asked for, bounded by the configuration's length."""
-    return max(1, min(asked, cfg.steps))
+def steps_per_launch_for(cfg, asked: int, calls: int = 0) -> int:
+    """Decode steps per br_step call.  What was asked for, if anything; else 16, or, when the timed
+    region has too few calls to walk one configuration length at 16 steps per call, the number
+    (at most 32) with which `calls` calls cover the configuration's steps exactly once, the
+    rotating sets taking one stretch of the trajectory each."""
+    if asked > 0:
+        return max(1, min(asked, cfg.steps))
+    if calls > 0 and calls * 16 < cfg.steps:
+        return max(1, min(32, -(-cfg.steps // calls)))
+    return 16
 
 
 # ----------------------------------------------------------------------------- CPU arm
@@ -271,8 +290,8 @@ def run_reference(args):
     import oracle
     cfg = wlm.get_config("c3")
     n_inst = 32
-    spl = steps_per_launch_for(cfg, args.steps_per_launch)
-    steps = min(args.steps, max(1, (cfg.steps - spl * args.warmup) // spl))
+    spl = steps_per_launch_for(cfg, args.steps_per_launch, args.steps)
+    steps = args.steps
     wl = wlm.make_workload(cfg, n_instances=n_inst)
     orcs = [oracle.instance_from_workload(wl, i) for i in range(n_inst)]
     for _ in range(args.warmup * spl):
@@ -396,19 +415,19 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     step changes along a configuration's trajectory (c3 starts with half-empty workers and a full
     queue, so its first ~80 steps admit several times more requests than the rest), so the sets
     start at evenly spaced points of the trajectory and the timed region is a stratified sample of
-    it (the whole of it when launches * spl reaches sets * configuration length).  Before every
-    repeat the sets return to their starting snapshots and one untimed call per set runs;
-    `warmup` untimed calls precede the first repeat."""
+    it (the whole of it, step 0 included, when launches * spl reaches sets * configuration length:
+    the default arguments do that for c3).  Before every repeat the sets return to their starting
+    snapshots; `warmup` untimed calls precede the first repeat."""
     cfg = wlm.get_config(wname)
     N = cfg.N if n_inst is None else n_inst
     per_inst_state = 4 * cfg.G * cfg.B + 8 * cfg.W + 4 * cfg.W + 64 * cfg.G
     n_sets = max(2, int(np.ceil(1.6 * L2_BYTES / (N * per_inst_state))))
-    n_sets = max(n_sets, int(np.ceil((launches + n_sets) * spl / cfg.steps)))
-    prime = n_sets
+    n_sets = max(n_sets, int(np.ceil(launches * spl / cfg.steps)))
+    prime = 0                                                 # the timed region starts at the sets' starting snapshots
     per_set = -(-(launches + prime) // n_sets)                # launches a set sees in one repeat
     span = per_set * spl
     room = max(0, cfg.steps - span)
-    starts = [int(j * room / max(1, n_sets - 1)) // spl * spl for j in range(n_sets)]
+    starts = [int(round(j * room / max(1, n_sets - 1))) // spl * spl for j in range(n_sets)]
     sets = RotatingSets(wname, N, n_sets, device, seed_offset=seed_offset, threads=threads,
                         probs_ring=probs_ring, spl=spl, start_steps=starts)
     starts = list(sets.start_steps)
@@ -499,7 +518,7 @@ def run_ours(args):
     # ---------------- headline: batched, several decode steps per launch ----------------
     wname = args.workload
     cfg = wlm.get_config(wname)
-    spl = steps_per_launch_for(cfg, args.steps_per_launch)
+    spl = steps_per_launch_for(cfg, args.steps_per_launch, args.steps)
     first, _ = shard_of(rank, world, cfg.N, 64)
     m = measure_batched(torch, wname, device, args.steps, args.warmup, spl, repeats=args.repeats,
                         threads=args.threads, seed_offset=first, dist=dist, sampler=ClockSampler(local))
@@ -520,8 +539,7 @@ def run_ours(args):
                    "instances_per_launch": N, "steps_per_launch": spl, "rotating_sets": m["n_sets"],
                    "repeats": args.repeats,
                    "timing": f"median of {args.repeats} repeats of the {args.steps}-call region (CUDA events; "
-                             f"before each repeat the sets return to their starting snapshots and one untimed "
-                             f"call per set runs)",
+                             f"before each repeat the sets return to their starting snapshots)",
                    "trajectory": m["trajectory"], "launches_before_timed": m["launches_before_timed"],
                    "l2": f"{m['n_sets']} instance sets stepped in rotation: data touched between two visits of a "
                          f"set exceeds the 126 MB L2; no instance runs past the configuration's {cfg.steps} steps",
@@ -783,10 +801,13 @@ def entry_points(torch, device, peak):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=60, help="br_step calls in the timed region")
+    ap.add_argument("--steps", type=int, default=124,
+                    help="br_step calls in the timed region (124 calls of 16 decode steps walk four instance sets "
+                         "through the whole 500-step configuration)")
     ap.add_argument("--warmup", type=int, default=10, help="untimed br_step calls before the first repeat")
-    ap.add_argument("--steps-per-launch", type=int, default=16,
-                    help="decode steps advanced by one br_step call (batch.n_steps)")
+    ap.add_argument("--steps-per-launch", type=int, default=0,
+                    help="decode steps advanced by one br_step call (batch.n_steps); 0 = 16, or with fewer than 32 "
+                         "calls in the timed region the number with which they cover the configuration exactly once")
     ap.add_argument("--repeats", type=int, default=7, help="repeats of the timed region; the median is reported")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
