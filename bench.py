@@ -552,14 +552,14 @@ def run_ours(args):
 
     if rank == 0 and world == 1 and not args.quick and wname == "c3":
         # the same workload with one decode step per launch (the form the latency path replays)
-        m1 = measure_batched(torch, wname, device, 400, 40, 1, repeats=5, threads=args.threads)
+        m1 = measure_batched(torch, wname, device, cfg.steps, 40, 1, repeats=5, threads=args.threads)   # one pass over the trajectory
         r1 = roofline_of(m1, wname, peak, peak_kind, clocks)
         line["single_step_launches"] = {"value": m1["value"], "unit": UNIT, "ms_per_step": m1["ms_per_launch"],
                                         "roofline": r1, "gpu_launches": m1["launches"], "repeats_ms": m1["repeats_ms"]}
         summary["c3_1_step_per_launch"] = brief(m1, r1)
         # two batches in one call (8,192 instances, one decode step): the second wave of thread blocks
         # fills the SMs that the first wave's short instances leave early
-        m2 = measure_batched(torch, wname, device, 200, 20, 1, repeats=5, threads=args.threads, n_inst=2 * N)
+        m2 = measure_batched(torch, wname, device, cfg.steps, 20, 1, repeats=5, threads=args.threads, n_inst=2 * N)
         line["single_step_launches_8192_instances"] = {
             "value": m2["value"], "unit": UNIT, "ms_per_step": m2["ms_per_launch"], "instances_per_launch": 2 * N,
             "us_per_4096_instance_steps": m2["us_per_launch"] / 2, "repeats_ms": m2["repeats_ms"],
