@@ -73,12 +73,13 @@ def test_c3_every_instance_every_array(spl):
     _compare_all(cfg, got, fin, ref, steps, range(cfg.N))
 
 
-def test_c4_every_instance_every_array():
+@pytest.mark.parametrize("spl", [1, 4])
+def test_c4_every_instance_every_array(spl):
     cfg = wlm.get_config("c4")
     steps = 20
     ref = oracle_batch("c4", cfg.N, steps)
     print(f"checker processes: {ref[5]}")
-    got, fin = _gpu_run(cfg, steps, 1)
+    got, fin = _gpu_run(cfg, steps, spl)
     _compare_all(cfg, got, fin, ref, steps, range(cfg.N))
 
 
