@@ -288,7 +288,8 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
     // scal: [0] queue length after routing, [1] admitted, [2] Stage-1 iterations,
     //       [3] Stage-2 pops, [4] status bits of the step, [5] status bits of the prologue,
     //       [6] requests that ended this step and were not prefetched, [7] prefetched ones,
-    //       [8] requests whose c_hat is refreshed at this step
+    //       [8] requests whose c_hat is refreshed at this step,
+    //       [9] set when requests that end were found before routing and did not fit the lists
 
     // ---- per-instance global rows ----
     const auto g_load = mk_span(reinterpret_cast<long long *>(a.ws.load) + (size_t)inst * G, G);
@@ -393,7 +394,9 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                         end_list[at] = (unsigned short)sa;
                     } else {                                         // list full: fix this slot up at once
                         atomicAdd(&sub_load[g], (unsigned)(g_base[sa] + k));
-                        g_base[sa] = kEmpty;
+                        // before routing the request still runs (the projection of this step counts
+                        // it): its slot is emptied in ADVANCE, found again through end_mask
+                        if (prefetch) scal[9] = 1; else g_base[sa] = kEmpty;
                     }
                 }
             }
@@ -1301,6 +1304,22 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                 g_base[sa] = kEmpty;
                 atomicAdd(&sub_load[sa / B], (unsigned)cur);
             }
+            if (have_pre && scal[9]) {
+                // more requests ended than the lists hold: the rest were subtracted when they were
+                // found, their slots are emptied here (the instance is one warp; the listed slots
+                // have been read by now)
+                __syncwarp();
+#pragma unroll 1
+                for (int idx = tid; idx < G * OW; idx += NT) {
+                    const int g = idx / OW, x = idx - g * OW;
+                    unsigned long long ended = end_mask[idx];
+                    while (ended) {
+                        const int j = __ffsll((long long)ended) - 1;
+                        ended &= ended - 1;
+                        g_base[g * B + 64 * x + j] = kEmpty;
+                    }
+                }
+            }
         }
         inst_sync();                                              // B3
 
@@ -1327,7 +1346,7 @@ __global__ void __maxnreg__((FP && HM > 0) ? 128 : 72) br_step_kernel(const Step
                     c[0] = (uint32_t)n_drop; c[1] = (uint32_t)scal[1]; c[2] = (uint32_t)scal[2]; c[3] = (uint32_t)scal[3];
                 }
                 if (a.out.status) a.out.status[orow] = scal[4] | scal[5];
-                scal[6] = 0; scal[7] = 0; scal[8] = 0;
+                scal[6] = 0; scal[7] = 0; scal[8] = 0; scal[9] = 0;
                 if (timing) {
                     t_phase[6] = (unsigned)clock64();
                     uint32_t *pc = a.out.phase_cycles + orow * 8;

@@ -292,3 +292,18 @@ def test_long_horizon_large_fleet_needs_more_than_48k_of_shared_memory():
                threads=256)
     run_parity(wlm.get_config("h80", G=64, W=1024, init_queue=1000, arrival=("const", 5.0)), 1, 8, check_every=4,
                graph=True)                             # the opt-in also happens while a graph is captured
+
+
+def test_more_requests_end_in_a_step_than_the_lists_hold():
+    # single-warp BR-H instances resolve the step's terminations before routing; with hundreds of
+    # requests ending at once the surplus must still count in that step's projection
+    for kw, threads, n, ls in [
+            (dict(G=47, B=72, W=36, H=8, init_active=42, init_queue=21, hazard=0.1, delta_T=7, gate=0.1, S_greedy=0,
+                  arrival=("const", 20.0)), 32, 3, 2),
+            (dict(G=32, B=72, W=256, H=16, init_active=48, init_queue=159, hazard=0.3, delta_T=2, gate=0.3,
+                  S_greedy=16, gamma=0.9, arrival=("const", 8.0)), 32, 8, 1),
+            (dict(G=8, B=64, W=1000, H=80, init_active=49, init_queue=737, hazard=0.3, delta_T=2, gate=0.3,
+                  S_greedy=0, beta=3.0, gamma=1.0, beta_ab=(1.0, 8.0), arrival=("const", 1.0)), 0, 5, 5),
+            (dict(G=32, B=64, W=256, H=0, init_active=60, init_queue=200, hazard=0.3, arrival=("const", 20.0)), 32, 4, 3)]:
+        cfg = wlm.get_config("c0", term_mode=1, score_mode=-1, **kw)
+        run_parity(cfg, n, 6 * ls, threads=threads, launch_steps=ls, check_every=1)
