@@ -36,11 +36,16 @@ UNIT = "instance-steps/s"
 METRICS = {
     "c3": "routing instance-steps/sec (batched BR-0, 4096 instances, G=32, W=256)",
     "c4": "routing instance-steps/sec (batched BR-H H=8, 1024 instances, G=64, W=1024)",
+    "h80": "routing instance-steps/sec (batched BR-H H=80 with perfect lookahead, 1024 instances, G=8, W=512)",
 }
 WORKLOADS = {
     "c3": "c3: BR-0 batched, 4096 instances/GPU, G=32, B=64, W=256, seeds 100..",
     "c4": "c4: BR-H H=8 batched, 1024 instances/GPU, G=64, B=64, W=1024, seeds 5000..",
+    "h80": "h80: BR-H H=80 (the paper's deployed horizon), perfect-lookahead predictor, requests with lifetimes, "
+           "1024 instances/GPU, G=8, B=64, W=512, seeds 9000..",
 }
+BATCH_INSTANCES = {"h80": 1024}          # workloads defined on one instance, benchmarked as a batch
+ARRIVALS_PER_STEP = {"c3": 10.0, "c4": 20.0, "h80": 0.7}
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -109,7 +114,9 @@ def algorithmic_bytes(cfg, edits_per_step: float, rho: float) -> float:
     one-byte refresh stamp); the extra byte is layout cost and is not counted here."""
     A, G, W, H = cfg.G * cfg.B, cfg.G, cfg.W, cfg.H
     b = 4.0 * A + 8.0 * W + 4.0 * W + 20.0 * G + 28.0 * G + 24.0 + 8.0 * edits_per_step
-    if H > 0:
+    if H > 0 and cfg.pred_mode == 1:
+        b += 4.0 * A + 8.0 * W           # perfect lookahead: the step each request ends at; output lengths of the queue
+    elif H > 0:
         b += 4.0 * A + 4.0 * H * A * rho + 4.0 * A / cfg.delta_T
     return b
 
@@ -455,7 +462,7 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     torch.cuda.empty_cache()
     ms = float(np.median(reps))
     # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
-    edits = float(2.0 * cnt[1] + (10.0 if wname == "c3" else 20.0))
+    edits = float(2.0 * cnt[1] + ARRIVALS_PER_STEP[wname])
     abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
     us_per_launch = 1e3 * ms / launches
     return dict(ms=ms, ms_per_launch=ms / launches, us_per_launch=us_per_launch, n_sets=n_sets, N=N, spl=spl,
@@ -467,7 +474,7 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
 
 
 def kernel_name(wname):
-    return "br_small_kernel<2,4>" if wname == "c3" else "br_step_kernel<true,8,2,1>"
+    return {"c3": "br_small_kernel<2,4>", "c4": "br_step_kernel<true,8,2,1>", "h80": "br_step_kernel<true,80,1,0>"}[wname]
 
 
 def roofline_of(m, wname, peak, peak_kind, clocks=None):
@@ -521,7 +528,8 @@ def run_ours(args):
     spl = steps_per_launch_for(cfg, args.steps_per_launch, args.steps)
     first, _ = shard_of(rank, world, cfg.N, 64)
     m = measure_batched(torch, wname, device, args.steps, args.warmup, spl, repeats=args.repeats,
-                        threads=args.threads, seed_offset=first, dist=dist, sampler=ClockSampler(local))
+                        threads=args.threads, seed_offset=first, dist=dist, sampler=ClockSampler(local),
+                        n_inst=BATCH_INSTANCES.get(wname))
     N = m["N"]
     value = world * m["value"]
     clocks = m["clocks"]
@@ -633,10 +641,10 @@ def extras(torch, device, args, peak, peak_kind, summary):
     # the deployed lookahead as a batch: 1,024 instances of the h80 workload (H = 80, G = 8, R_max = 4), 8 steps per launch
     try:
         mh = measure_batched(torch, "h80", device, 24, 4, 8, repeats=5, n_inst=1024)
+        rh = roofline_of(mh, "h80", peak, peak_kind)
         ex["h80_batched"] = {"value": mh["value"], "unit": UNIT, "ms_per_step": mh["ms_per_launch"], "steps_per_launch": 8,
-                             "instances_per_launch": 1024, "repeats_ms": mh["repeats_ms"]}
-        summary["h80_batched_1024_instances"] = {"us_per_decode_step": round(mh["us_per_launch"] / 8, 2),
-                                                 "inst_steps_per_s": round(mh["value"])}
+                             "instances_per_launch": 1024, "repeats_ms": mh["repeats_ms"], "roofline": rh}
+        summary["h80_batched_1024_instances"] = brief(mh, rh)
     except Exception as e:
         ex["h80_batched"] = {"error": repr(e)}
     # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
@@ -812,7 +820,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--threads", type=int, default=0, help="threads per instance (0 = library default)")
     ap.add_argument("--quick", action="store_true", help="headline measurement only")
-    ap.add_argument("--workload", default="c3", choices=["c3", "c4"],
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "h80"],
                     help="batched configuration timed as the headline (c4 is used for profiling the BR-H kernel)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
