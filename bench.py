@@ -45,7 +45,7 @@ WORKLOADS = {
            "1024 instances/GPU, G=8, B=64, W=512, seeds 9000..",
 }
 BATCH_INSTANCES = {"h80": 1024}          # workloads defined on one instance, benchmarked as a batch
-ARRIVALS_PER_STEP = {"c3": 10.0, "c4": 20.0, "h80": 0.7}
+ARRIVALS_PER_STEP = {"c3": 10.0, "c4": 20.0, "h80": 0.7, "c2": 8.0}
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -463,7 +463,9 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
     ms = float(np.median(reps))
     # edits per instance-step: admissions + terminations (= admissions in steady state) + arrivals
     edits = float(2.0 * cnt[1] + ARRIVALS_PER_STEP[wname])
-    abytes = algorithmic_bytes(cfg, edits, 1.0 / cfg.delta_T if cfg.H > 0 else 0.0) * N * spl
+    # share of the classifier rows a step needs: every row when terminations are drawn from them
+    rho = 0.0 if cfg.H == 0 else (1.0 if cfg.term_mode == 2 else 1.0 / cfg.delta_T)
+    abytes = algorithmic_bytes(cfg, edits, rho) * N * spl
     us_per_launch = 1e3 * ms / launches
     return dict(ms=ms, ms_per_launch=ms / launches, us_per_launch=us_per_launch, n_sets=n_sets, N=N, spl=spl,
                 launches_before_timed=launches_before,
@@ -474,7 +476,8 @@ def measure_batched(torch, wname, device, launches, warmup, spl, repeats=5, thre
 
 
 def kernel_name(wname):
-    return {"c3": "br_small_kernel<2,4>", "c4": "br_step_kernel<true,8,2,1>", "h80": "br_step_kernel<true,80,1,0>"}[wname]
+    return {"c3": "br_small_kernel<2,4>", "c4": "br_step_kernel<true,8,2,1>", "h80": "br_step_kernel<true,80,1,0>",
+            "c2": "br_step_kernel<true,4,1,0>"}[wname]
 
 
 def roofline_of(m, wname, peak, peak_kind, clocks=None):
@@ -647,6 +650,16 @@ def extras(torch, device, args, peak, peak_kind, summary):
         summary["h80_batched_1024_instances"] = brief(mh, rh)
     except Exception as e:
         ex["h80_batched"] = {"error": repr(e)}
+    # the c2 shape as a batch (2,048 instances, H = 4, terminations drawn from the classifier rows, so every
+    # row is read every step): the most HBM-like of the step workloads
+    try:
+        m2 = measure_batched(torch, "c2", device, 60, 6, 4, repeats=5, n_inst=2048)
+        r2 = roofline_of(m2, "c2", peak, peak_kind)
+        ex["c2_batched"] = {"value": m2["value"], "unit": UNIT, "ms_per_step": m2["ms_per_launch"], "steps_per_launch": 4,
+                            "instances_per_launch": 2048, "repeats_ms": m2["repeats_ms"], "roofline": r2}
+        summary["c2_batched_2048_instances"] = brief(m2, r2)
+    except Exception as e:
+        ex["c2_batched"] = {"error": repr(e)}
     # the stand-alone entry points: F-score matrix, pool-bypass dispatch, exact subset solver
     try:
         ex["entry_points"] = entry_points(torch, device, peak)
